@@ -1,0 +1,154 @@
+/*
+ * i8ops — int8 GEMM, NHWC conv2d and batched/skinny GEMM for NVIDIA B200 (sm_100a), each with a fused
+ * read-out epilogue (int32 bias, optional ReLU, fixed-point scale, saturating narrow to int8).
+ *
+ * These are the tensor operations that the Autocomp paper (arXiv 2505.18574) optimises on a
+ * Gemmini-style accelerator: 8-bit integer operands accumulated in 32 bits (Evaluation, "Gemmini
+ * Evaluation"), computed tile by tile as  move-in -> matrix unit -> accumulator -> scaled move-out
+ * (Background, the figure that sets CPU code beside accelerator code; Gemmini ISA description in the
+ * Prompts appendix).  Here the scratchpad is shared memory fed by TMA, the matrix unit is
+ * tcgen05.mma kind::i8, the accumulator is tensor memory, and the move-out is the fused epilogue.
+ *
+ * Epilogue, applied to every accumulator acc (exact, evaluated in 64-bit integers):
+ *     t   = acc + bias[n]                      (bias == NULL means 0; ISA description: C = A*B + bias)
+ *     t   = max(t, 0)            if relu       (RELU activation of the ISA's execute configuration)
+ *     u   = floor((t * mult[n] + r) / 2^shift[n]),   r = 2^(shift-1) if shift >= 1 else 0
+ *     out = min(127, max(-128, u))             (reading the accumulator as scaled-down input-type
+ *                                               data, ISA description continued)
+ * The paper shows the scale only as a float argument; this library fixes it as the multiplier/shift
+ * pair above (round half toward +infinity).  mult = 1, shift = 0, no bias, no ReLU reproduces the
+ * saturating C = A*B of the paper's printed Gemmini GEMM listing.
+ *
+ * Conventions for every compute entry point below
+ *   - All tensor, bias, mult and shift pointers are DEVICE pointers owned by the caller (the *_host
+ *     variants take HOST pointers and say so).  Inputs are never written.  The output must not
+ *     overlap any input.
+ *   - Strides are in elements (= bytes for the int8 tensors).
+ *   - mult / shift hold one entry (per_channel == 0) or N entries indexed by output channel
+ *     (per_channel != 0).  Any int32 multiplier is legal; every shift must lie in [0, 31] (not
+ *     checked on the device: the caller guarantees it, the host variants check it).
+ *   - Contract on magnitudes: acc + bias must fit in int32 (guaranteed for K <= 65536 with
+ *     |bias| < 2^30); behaviour beyond that is unspecified.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - The return value is an i8_status for errors the host can detect before launching; nothing is
+ *     launched when it is non-zero.  The library never throws, aborts or exits.
+ *   - Every wait inside the kernels is bounded.  If one ever expires the kernel stops early, leaves
+ *     the rest of the output unwritten and records the fact; i8ops_last_device_status() reports it.
+ */
+#ifndef I8OPS_H
+#define I8OPS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    I8_OK = 0,
+    I8_ERR_NULL = 1,        /* a required pointer is NULL */
+    I8_ERR_SHAPE = 2,       /* a negative extent, or a convolution with an empty output */
+    I8_ERR_STRIDE = 3,      /* neither stride of an operand is 1, or a leading dimension is too small */
+    I8_ERR_ALIGN = 4,       /* reserved: misaligned operands are served by the generic kernel instead */
+    I8_ERR_RANGE = 5,       /* K > 65536, or (host variants) a shift outside [0, 31] */
+    I8_ERR_UNSUPPORTED = 6, /* stride or padding outside what the convolution supports */
+    I8_ERR_CUDA = 7,        /* a CUDA runtime or driver call failed; see i8ops_last_cuda_error() */
+    I8_ERR_TIMEOUT = 8      /* a bounded wait inside a kernel expired (device status only) */
+} i8_status;
+
+/* Which kernel family served the most recent compute call of this thread (for tests and tuning). */
+typedef enum {
+    I8_PATH_NONE = 0,       /* nothing launched (empty problem or error) */
+    I8_PATH_GENERIC = 1,    /* one-thread-per-output kernel: any strides, any alignment */
+    I8_PATH_TENSOR = 2,     /* TMA -> shared memory ring -> tcgen05.mma kind::i8 -> tensor memory -> epilogue */
+    I8_PATH_SMALL = 3       /* small-tile tensor path: resident B / paired 64x64 problems */
+} i8_path;
+
+/*
+ * C[m*ldc + n] = epilogue( sum_k A[m*a_rs + k*a_cs] * B[k*b_rs + n*b_cs] ),  0 <= m < M, 0 <= n < N.
+ * (The product of the paper's matrix-multiplication figure; int8 x int8 accumulated in int32.)
+ *   A, B   device, int8.  Exactly one of (a_rs, a_cs) and one of (b_rs, b_cs) must be 1; the other is the
+ *          leading dimension (>= the extent it strides over).  Row-major A is (a_rs = lda, a_cs = 1);
+ *          column-major B is (b_rs = 1, b_cs = ldb).
+ *   C      device, int8, row-major, ldc >= N.
+ *   bias   device, int32[N], or NULL.
+ *   mult, shift, per_channel, relu   see the epilogue above.
+ * The tensor path needs both operands K-contiguous (a_cs == 1, b_rs == 1) with 16-byte aligned base
+ * addresses and leading dimensions; anything else is computed by the generic kernel, same results.
+ * Errors: I8_ERR_NULL, I8_ERR_SHAPE (negative M, N or K), I8_ERR_STRIDE, I8_ERR_RANGE, I8_ERR_CUDA.
+ * M == 0 or N == 0 returns I8_OK and launches nothing; K == 0 yields epilogue(0).
+ */
+int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs,
+            const int8_t* B, int64_t b_rs, int64_t b_cs,
+            int8_t* C, int64_t ldc,
+            const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
+            int M, int N, int K, int relu, void* stream);
+
+/*
+ * `batch` independent products (the paper's fine-grained linear algebra: many small, low-reuse
+ * products, Evaluation "Fine-Grained Linear Algebra"; also its column-dominant GEMM shapes).
+ * Problem b uses A + b*a_bs, B + b*b_bs, C + b*c_bs and bias + b*bias_bs (bias_bs == 0: one bias
+ * shared by all problems); mult/shift are shared by all problems.  Other arguments as gemm_i8.
+ * Errors as gemm_i8, plus I8_ERR_SHAPE for a negative batch.
+ */
+int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs,
+                    const int8_t* B, int64_t b_rs, int64_t b_cs, int64_t b_bs,
+                    int8_t* C, int64_t ldc, int64_t c_bs,
+                    const int32_t* bias, int64_t bias_bs,
+                    const int32_t* mult, const int32_t* shift, int per_channel,
+                    int batch, int M, int N, int K, int relu, void* stream);
+
+/*
+ * y[n][p][q][k] = epilogue( sum_{r,s,c} x[n][p*stride_h - pad_h + r][q*stride_w - pad_w + s][c] * w[k][r][s][c] )
+ * (the paper's ResNet-50 convolution benchmarks, Evaluation "Convolution", lowered to an implicit GEMM
+ * with M = N*P*Q, N = K filters, K = R*S*C).  Cross-correlation (no kernel flip); taps outside the image
+ * contribute 0; dilation 1, groups 1.
+ *   x  device int8 [N][H][W][C] (NHWC, dense);  w  device int8 [K][R][S][C] (dense);
+ *   y  device int8 [N][P][Q][K] (dense),  P = floor((H + 2*pad_h - R)/stride_h) + 1, Q likewise.
+ *   bias/mult/shift indexed by filter k.
+ * Errors: I8_ERR_NULL, I8_ERR_SHAPE (a non-positive extent or an empty output), I8_ERR_UNSUPPORTED
+ * (stride < 1, pad < 0), I8_ERR_RANGE (R*S*C > 65536), I8_ERR_CUDA.
+ */
+int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y,
+              const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
+              int N, int H, int W, int C, int K, int R, int S,
+              int stride_h, int stride_w, int pad_h, int pad_w, int relu, void* stream);
+
+/*
+ * Host-buffer variants: every pointer is HOST memory (pinned memory makes the copies asynchronous).
+ * The call copies the operands to a device workspace that the library keeps per device (grown with
+ * cudaMalloc when a larger problem arrives, never shrunk), runs the same kernels, copies the result
+ * back and synchronises `stream` before returning.  They also check every shift (I8_ERR_RANGE).
+ * Tight layouts only: A row-major [M][K], B column-major (K contiguous, [N][K]), C row-major [M][N].
+ */
+int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C,
+                 const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
+                 int M, int N, int K, int relu, void* stream);
+
+/* Human-readable name of an i8_status. */
+const char* i8_status_string(int status);
+
+/* Synchronises `stream`, then returns I8_OK, I8_ERR_TIMEOUT if a bounded wait expired in any kernel of
+ * this library on the current device since the last call, or I8_ERR_CUDA.  Clears the record. */
+int i8ops_last_device_status(void* stream);
+
+/* cudaError_t of the most recent failed CUDA call made by this library on this thread (0 if none). */
+int i8ops_last_cuda_error(void);
+
+/* i8_path of the most recent compute call made by this thread. */
+int i8ops_last_path(void);
+
+/* Restrict dispatch: 0 = automatic (default), 1 = always the generic kernel, 2 = tensor paths whenever
+ * their layout requirements hold (also for tiny problems).  Returns the previous setting. */
+int i8ops_set_path(int mode);
+
+/* Upper limit, in milliseconds, for any single wait inside a kernel (default 2000). */
+void i8ops_set_wait_limit_ms(int ms);
+
+/* Library ABI version (bumped when a signature changes). */
+int i8ops_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* I8OPS_H */

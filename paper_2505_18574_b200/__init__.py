@@ -1,0 +1,13 @@
+"""i8ops for B200: int8 GEMM / conv2d / batched GEMM with a fused requantising epilogue.
+
+``binding`` holds the ctypes front end of the C-ABI library ``libi8ops.so`` (argument marshalling only:
+every step of the computation runs in the CUDA kernels).  ``inputs`` holds the seeded synthetic workloads.
+``build`` compiles the library with nvcc for sm_100a.
+"""
+from .binding import (I8Error, batched_gemm_i8, conv2d_i8, gemm_i8, gemm_i8_host, last_device_status, last_path,
+                      lib, set_path, set_wait_limit_ms, status_string, PATH_GENERIC, PATH_NONE, PATH_SMALL,
+                      PATH_TENSOR)
+
+__all__ = ["I8Error", "batched_gemm_i8", "conv2d_i8", "gemm_i8", "gemm_i8_host", "last_device_status", "last_path",
+           "lib", "set_path", "set_wait_limit_ms", "status_string", "PATH_GENERIC", "PATH_NONE", "PATH_SMALL",
+           "PATH_TENSOR"]

@@ -1,0 +1,147 @@
+"""ctypes binding of ``libi8ops.so`` with the same entry-point names as ``include/i8ops.h``.
+
+Only argument marshalling happens here: tensors are torch CUDA tensors (torch is used for device memory
+and streams), from which pointers, extents and strides are read and passed to the C ABI.  There is no
+fallback: if the library is missing or a call reports an error, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libi8ops.so")
+_lib = None
+
+PATH_NONE, PATH_GENERIC, PATH_TENSOR, PATH_SMALL = 0, 1, 2, 3
+
+_vp = ctypes.c_void_p
+_i64 = ctypes.c_int64
+_int = ctypes.c_int
+
+# name -> (restype, argtypes); every symbol that include/i8ops.h declares
+SIGNATURES = {
+    "gemm_i8": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
+    "batched_gemm_i8": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _int,
+                               _int, _int, _int, _int, _int, _vp]),
+    "conv2d_i8": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int] + [_int] * 12 + [_vp]),
+    "gemm_i8_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
+    "i8_status_string": (ctypes.c_char_p, [_int]),
+    "i8ops_last_device_status": (_int, [_vp]),
+    "i8ops_last_cuda_error": (_int, []),
+    "i8ops_last_path": (_int, []),
+    "i8ops_set_path": (_int, [_int]),
+    "i8ops_set_wait_limit_ms": (None, [_int]),
+    "i8ops_version": (_int, []),
+}
+
+
+class I8Error(RuntimeError):
+    """A call into libi8ops returned a non-zero status."""
+
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: i8_status {status} ({status_string(status)})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libi8ops.so`` (built by ``python -m paper_2505_18574_b200.build``); raise if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2505_18574_b200.build` "
+                               "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().i8_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise I8Error(status, where)
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return getattr(stream, "cuda_stream", stream)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def gemm_i8(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:
+    """C = epilogue(A . B).  A: (M, K) int8 view, B: (K, N) int8 view (pass ``Bt.t()`` for a column-major B
+    stored as (N, K)), C: (M, N) int8 with unit column stride; bias int32 [N] or None; mult/shift int32 [1] or [N]."""
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2 and tuple(C.shape) == (M, N) and (C.stride(1) == 1 or N <= 1)
+    st = lib().gemm_i8(_ptr(A), A.stride(0), A.stride(1), _ptr(B), B.stride(0), B.stride(1), _ptr(C), C.stride(0),
+                       _ptr(bias), _ptr(mult), _ptr(shift), int(per_channel), M, N, K, int(relu), _stream_ptr(stream))
+    _check(st, "gemm_i8")
+
+
+def batched_gemm_i8(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:
+    """A: (batch, M, K), B: (batch, K, N), C: (batch, M, N) int8 views; bias int32 (batch, N), (N,) or None."""
+    batch, M, K = A.shape
+    _, K2, N = B.shape
+    assert K == K2 and tuple(C.shape) == (batch, M, N) and (C.stride(2) == 1 or N <= 1)
+    bias_bs = 0
+    if bias is not None and bias.dim() == 2:
+        bias_bs = bias.stride(0)
+    st = lib().batched_gemm_i8(_ptr(A), A.stride(1), A.stride(2), A.stride(0), _ptr(B), B.stride(1), B.stride(2),
+                               B.stride(0), _ptr(C), C.stride(1), C.stride(0), _ptr(bias), bias_bs, _ptr(mult),
+                               _ptr(shift), int(per_channel), batch, M, N, K, int(relu), _stream_ptr(stream))
+    _check(st, "batched_gemm_i8")
+
+
+def conv2d_i8(x, w, y, bias, mult, shift, per_channel: int, relu: int, stride=(1, 1), pad=(0, 0), stream=None) -> None:
+    """x: (N, H, W, C), w: (K, R, S, C), y: (N, P, Q, K), all dense int8."""
+    N, H, W, C = x.shape
+    K, R, S, C2 = w.shape
+    assert C == C2 and x.is_contiguous() and w.is_contiguous() and y.is_contiguous()
+    st = lib().conv2d_i8(_ptr(x), _ptr(w), _ptr(y), _ptr(bias), _ptr(mult), _ptr(shift), int(per_channel),
+                         N, H, W, C, K, R, S, int(stride[0]), int(stride[1]), int(pad[0]), int(pad[1]), int(relu),
+                         _stream_ptr(stream))
+    _check(st, "conv2d_i8")
+
+
+def gemm_i8_host(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:
+    """Host-buffer GEMM: A (M, K), B stored column-major as (N, K), C (M, N), all contiguous host tensors or
+    numpy arrays (anything with ``data_ptr()`` or ``ctypes.data``); copies in, computes on the GPU, copies out."""
+    def hp(a):
+        if a is None:
+            return None
+        return a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data
+    M, K = A.shape
+    N = B.shape[0]
+    st = lib().gemm_i8_host(hp(A), hp(B), hp(C), hp(bias), hp(mult), hp(shift), int(per_channel), M, N, K, int(relu),
+                            _stream_ptr(stream))
+    _check(st, "gemm_i8_host")
+
+
+def last_device_status(stream=None) -> int:
+    return lib().i8ops_last_device_status(_stream_ptr(stream))
+
+
+def last_path() -> int:
+    return lib().i8ops_last_path()
+
+
+def set_path(mode: int) -> int:
+    return lib().i8ops_set_path(int(mode))
+
+
+def set_wait_limit_ms(ms: int) -> None:
+    lib().i8ops_set_wait_limit_ms(int(ms))

@@ -1,0 +1,364 @@
+// C-ABI entry points of i8ops: argument validation, dispatch, tensor-map construction, launches.
+// Everything that computes runs in the kernels included below; the host code only marshals.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "../../include/i8ops.h"
+#include "gemm_tc.cuh"
+#include "generic.cuh"
+
+namespace i8 {
+
+// ------------------------------------------------------------------------------------------------ state
+__device__ unsigned g_dev_status = 0;   // first bounded-wait expiry since the last query (0 = none)
+
+constexpr int MAX_DEVICES = 64;
+
+struct DeviceCtx {
+    bool ready = false;
+    int sm_count = 0;
+    unsigned* dev_status = nullptr;   // device address of g_dev_status
+    bool attr_set[16] = {};           // dynamic shared-memory opt-in done, per kernel instance
+    void* ws = nullptr;               // workspace of the host-buffer variants
+    size_t ws_bytes = 0;
+};
+
+static DeviceCtx g_ctx[MAX_DEVICES];
+static std::mutex g_mutex;
+static int g_path_mode = 0;                      // 0 auto, 1 generic only, 2 tensor whenever legal
+static uint64_t g_wait_limit_ns = 2000ull * 1000 * 1000;
+static int g_force_bn = -1;                      // tuning override from the environment (I8OPS_FORCE_BN)
+
+static thread_local int t_last_path = I8_PATH_NONE;
+static thread_local int t_last_cuda = 0;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode_tiled = nullptr;
+
+static int cuda_fail(cudaError_t e) {
+    t_last_cuda = (int)e;
+    return I8_ERR_CUDA;
+}
+
+#define CUDA_TRY(expr)                                   \
+    do {                                                 \
+        cudaError_t _e = (expr);                         \
+        if (_e != cudaSuccess) return cuda_fail(_e);     \
+    } while (0)
+
+// Per-device set-up on first use: SM count, address of the status word, driver entry point.
+static int get_ctx(DeviceCtx** out) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return cuda_fail(cudaErrorInvalidDevice);
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx& c = g_ctx[dev];
+    if (!c.ready) {
+        CUDA_TRY(cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        CUDA_TRY(cudaGetSymbolAddress((void**)&c.dev_status, g_dev_status));
+        if (!g_encode_tiled) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult q;
+            CUDA_TRY(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &q));
+            if (q != cudaDriverEntryPointSuccess || !fn) return cuda_fail(cudaErrorNotSupported);
+            g_encode_tiled = (EncodeTiledFn)fn;
+        }
+        const char* bn = getenv("I8OPS_FORCE_BN");
+        if (bn) g_force_bn = atoi(bn);
+        c.ready = true;
+    }
+    *out = &c;
+    return I8_OK;
+}
+
+// 2-D or 3-D byte tensor, innermost dimension contiguous, 128-byte swizzle, zero fill outside.
+static int make_tmap(CUtensorMap* tm, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                     const uint32_t* box, CUtensorMapSwizzle swz) {
+    cuuint64_t gdim[5], gstr[4];
+    cuuint32_t bx[5], es[5];
+    for (int i = 0; i < rank; i++) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i + 1 < rank; i++) gstr[i] = strides_bytes[i];
+    CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bx, es,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { t_last_cuda = (int)cudaErrorInvalidValue; return I8_ERR_CUDA; }
+    return I8_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------------------------------------ launches
+template <int BN, int STAGES>
+static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUtensorMap& tmB, GemmTcParams& p,
+                     cudaStream_t st) {
+    using L = TcSmem<BN, STAGES>;
+    auto kern = gemm_i8_tc_kernel<BN, STAGES>;
+    if (!ctx->attr_set[slot]) {
+        CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES));
+        ctx->attr_set[slot] = true;
+    }
+    const int grid = p.sched.num_tiles < ctx->sm_count ? p.sched.num_tiles : ctx->sm_count;
+    kern<<<grid, TC_THREADS, L::DYN_BYTES, st>>>(tmA, tmB, p);
+    CUDA_TRY(cudaGetLastError());
+    return I8_OK;
+}
+
+// Tile width: model each K block as operand-delivery bound (256 + 2*BN cycles) and pick the width with the
+// fewest total cycles over all waves; ties go to the wider tile.
+static int choose_bn(int M, int N, int sm_count) {
+    if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256) return g_force_bn;
+    const int cands[3] = {256, 128, 64};
+    int best = 64;
+    double best_cost = 1e300;
+    const int m_tiles = (M + BM - 1) / BM;
+    for (int i = 0; i < 3; i++) {
+        const int bn = cands[i];
+        if (bn > 64 && bn - 64 >= ((N + 63) / 64) * 64) continue;   // tile mostly empty
+        const int64_t tiles = (int64_t)m_tiles * ((N + bn - 1) / bn);
+        const int64_t waves = (tiles + sm_count - 1) / sm_count;
+        const double cost = (double)waves * (256.0 + 2.0 * bn);
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = bn; }
+    }
+    return best;
+}
+
+static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
+                       const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
+                       int K, int relu, cudaStream_t st) {
+    const int bn = choose_bn(M, N, ctx->sm_count);
+    CUtensorMap tmA, tmB;
+    {
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
+        const uint64_t str[1] = {(uint64_t)lda};
+        const uint32_t box[2] = {BK, BM};
+        int rc = make_tmap(&tmA, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (rc) return rc;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
+        const uint64_t str[1] = {(uint64_t)ldb};
+        const uint32_t box[2] = {BK, (uint32_t)bn};
+        int rc = make_tmap(&tmB, B, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (rc) return rc;
+    }
+    GemmTcParams p;
+    p.C = C; p.ldc = ldc; p.bias = bias; p.mult = mult; p.shift = shift;
+    p.per_channel = per_channel; p.relu = relu; p.M = M; p.N = N; p.K = K;
+    p.c_vec_ok = aligned16(C) && (ldc % 16 == 0);
+    p.sched.m_tiles = (M + BM - 1) / BM;
+    p.sched.n_tiles = (N + bn - 1) / bn;
+    p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
+    p.sched.group_m = 16;
+    p.wait_limit_ns = g_wait_limit_ns;
+    p.dev_status = ctx->dev_status;
+    switch (bn) {
+        case 256: return launch_tc<256, 4>(ctx, 0, tmA, tmB, p, st);
+        case 128: return launch_tc<128, 6>(ctx, 1, tmA, tmB, p, st);
+        default:  return launch_tc<64, 8>(ctx, 2, tmA, tmB, p, st);
+    }
+}
+
+static int run_gemm_generic(const GenericGemmParams& p, cudaStream_t st) {
+    const int64_t total = (int64_t)p.batch * p.M * p.N;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    gemm_i8_generic_kernel<<<(int)blocks, 256, 0, st>>>(p);
+    CUDA_TRY(cudaGetLastError());
+    return I8_OK;
+}
+
+// One operand's strides: the unit stride picks the contiguous axis, the other must span it.
+static bool strides_ok(int64_t rs, int64_t cs, int rows, int cols) {
+    if (rs < 0 || cs < 0) return false;
+    if (cs == 1 && (rs >= cols || rows <= 1)) return true;
+    if (rs == 1 && (cs >= rows || cols <= 1)) return true;
+    return false;
+}
+
+static int validate_gemm(const void* A, int64_t a_rs, int64_t a_cs, const void* B, int64_t b_rs, int64_t b_cs, const void* C,
+                         int64_t ldc, const void* mult, const void* shift, int M, int N, int K) {
+    if (M < 0 || N < 0 || K < 0) return I8_ERR_SHAPE;
+    if (K > 65536) return I8_ERR_RANGE;
+    if (M == 0 || N == 0) return I8_OK;
+    if (!C || !mult || !shift || (K > 0 && (!A || !B))) return I8_ERR_NULL;
+    if (!strides_ok(a_rs, a_cs, M, K) || !strides_ok(b_rs, b_cs, K, N)) return I8_ERR_STRIDE;
+    if (ldc < N) return I8_ERR_STRIDE;
+    return I8_OK;
+}
+
+}  // namespace i8
+
+using namespace i8;
+
+// ================================================================================================ C ABI
+extern "C" {
+
+int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_t b_rs, int64_t b_cs, int8_t* C, int64_t ldc,
+            const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N, int K, int relu,
+            void* stream) {
+    t_last_path = I8_PATH_NONE;
+    int rc = validate_gemm(A, a_rs, a_cs, B, b_rs, b_cs, C, ldc, mult, shift, M, N, K);
+    if (rc) return rc;
+    if (M == 0 || N == 0) return I8_OK;
+    DeviceCtx* ctx = nullptr;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool tc_legal = K >= 1 && a_cs == 1 && b_rs == 1 && aligned16(A) && aligned16(B) && a_rs % 16 == 0 &&
+                          b_cs % 16 == 0 && a_rs >= K && b_cs >= K;
+    if (tc_legal && g_path_mode != 1) {
+        rc = run_gemm_tc(ctx, A, a_rs, B, b_cs, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
+        if (rc == I8_OK) t_last_path = I8_PATH_TENSOR;
+        return rc;
+    }
+    GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, C, ldc, 0, bias, 0, mult, shift, per_channel, relu, 1, M, N, K};
+    rc = run_gemm_generic(g, st);
+    if (rc == I8_OK) t_last_path = I8_PATH_GENERIC;
+    return rc;
+}
+
+int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs, const int8_t* B, int64_t b_rs, int64_t b_cs,
+                    int64_t b_bs, int8_t* C, int64_t ldc, int64_t c_bs, const int32_t* bias, int64_t bias_bs,
+                    const int32_t* mult, const int32_t* shift, int per_channel, int batch, int M, int N, int K, int relu,
+                    void* stream) {
+    t_last_path = I8_PATH_NONE;
+    if (batch < 0) return I8_ERR_SHAPE;
+    int rc = validate_gemm(A, a_rs, a_cs, B, b_rs, b_cs, C, ldc, mult, shift, M, N, K);
+    if (rc) return rc;
+    if (a_bs < 0 || b_bs < 0 || c_bs < 0 || bias_bs < 0) return I8_ERR_STRIDE;
+    if (batch == 0 || M == 0 || N == 0) return I8_OK;
+    DeviceCtx* ctx = nullptr;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    GenericGemmParams g{A, a_rs, a_cs, a_bs, B, b_rs, b_cs, b_bs, C, ldc, c_bs, bias, bias_bs, mult, shift, per_channel, relu,
+                        batch, M, N, K};
+    rc = run_gemm_generic(g, st);
+    if (rc == I8_OK) t_last_path = I8_PATH_GENERIC;
+    return rc;
+}
+
+int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, const int32_t* mult, const int32_t* shift,
+              int per_channel, int N, int H, int W, int C, int K, int R, int S, int stride_h, int stride_w, int pad_h,
+              int pad_w, int relu, void* stream) {
+    t_last_path = I8_PATH_NONE;
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || K <= 0 || R <= 0 || S <= 0) return I8_ERR_SHAPE;
+    if (stride_h < 1 || stride_w < 1 || pad_h < 0 || pad_w < 0) return I8_ERR_UNSUPPORTED;
+    if (H + 2 * pad_h < R || W + 2 * pad_w < S) return I8_ERR_SHAPE;
+    if ((int64_t)R * S * C > 65536) return I8_ERR_RANGE;
+    if (!x || !w || !y || !mult || !shift) return I8_ERR_NULL;
+    const int P = (H + 2 * pad_h - R) / stride_h + 1;
+    const int Q = (W + 2 * pad_w - S) / stride_w + 1;
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    GenericConvParams g{x, w, y, bias, mult, shift, per_channel, relu, N, H, W, C, K, R, S, P, Q, stride_h, stride_w, pad_h, pad_w};
+    const int64_t total = (int64_t)N * P * Q * K;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    conv2d_i8_generic_kernel<<<(int)blocks, 256, 0, st>>>(g);
+    CUDA_TRY(cudaGetLastError());
+    t_last_path = I8_PATH_GENERIC;
+    return I8_OK;
+}
+
+int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C, const int32_t* bias, const int32_t* mult, const int32_t* shift,
+                 int per_channel, int M, int N, int K, int relu, void* stream) {
+    t_last_path = I8_PATH_NONE;
+    if (M < 0 || N < 0 || K < 0) return I8_ERR_SHAPE;
+    if (K > 65536) return I8_ERR_RANGE;
+    if (M == 0 || N == 0) return I8_OK;
+    if (!C || !mult || !shift || (K > 0 && (!A || !B))) return I8_ERR_NULL;
+    const int nq = per_channel ? N : 1;
+    for (int i = 0; i < nq; i++)
+        if (shift[i] < 0 || shift[i] > 31) return I8_ERR_RANGE;
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t szA = up((size_t)M * K), szB = up((size_t)N * K), szC = up((size_t)M * N);
+    const size_t szV = up((size_t)N * 4);
+    const size_t need = szA + szB + szC + 3 * szV;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (ctx->ws_bytes < need) {
+            if (ctx->ws) { CUDA_TRY(cudaDeviceSynchronize()); CUDA_TRY(cudaFree(ctx->ws)); ctx->ws = nullptr; ctx->ws_bytes = 0; }
+            CUDA_TRY(cudaMalloc(&ctx->ws, need));
+            ctx->ws_bytes = need;
+        }
+    }
+    uint8_t* base = (uint8_t*)ctx->ws;
+    int8_t* dA = (int8_t*)base; int8_t* dB = (int8_t*)(base + szA); int8_t* dC = (int8_t*)(base + szA + szB);
+    int32_t* dbias = (int32_t*)(base + szA + szB + szC);
+    int32_t* dmult = (int32_t*)((uint8_t*)dbias + szV);
+    int32_t* dshift = (int32_t*)((uint8_t*)dmult + szV);
+    if (K > 0) {
+        CUDA_TRY(cudaMemcpyAsync(dA, A, (size_t)M * K, cudaMemcpyHostToDevice, st));
+        CUDA_TRY(cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, st));
+    }
+    if (bias) CUDA_TRY(cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(dmult, mult, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(dshift, shift, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
+    rc = gemm_i8(dA, K, 1, dB, 1, K, dC, N, bias ? dbias : nullptr, dmult, dshift, per_channel, M, N, K, relu, stream);
+    if (rc) return rc;
+    CUDA_TRY(cudaMemcpyAsync(C, dC, (size_t)M * N, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return I8_OK;
+}
+
+const char* i8_status_string(int status) {
+    switch (status) {
+        case I8_OK: return "ok";
+        case I8_ERR_NULL: return "null pointer";
+        case I8_ERR_SHAPE: return "bad shape";
+        case I8_ERR_STRIDE: return "bad stride";
+        case I8_ERR_ALIGN: return "bad alignment";
+        case I8_ERR_RANGE: return "value out of range";
+        case I8_ERR_UNSUPPORTED: return "unsupported";
+        case I8_ERR_CUDA: return "CUDA call failed";
+        case I8_ERR_TIMEOUT: return "a bounded wait expired inside a kernel";
+        default: return "unknown status";
+    }
+}
+
+int i8ops_last_device_status(void* stream) {
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    unsigned v = 0;
+    CUDA_TRY(cudaMemcpy(&v, ctx->dev_status, sizeof(v), cudaMemcpyDeviceToHost));
+    if (v != 0) {
+        const unsigned zero = 0;
+        CUDA_TRY(cudaMemcpy(ctx->dev_status, &zero, sizeof(zero), cudaMemcpyHostToDevice));
+        return I8_ERR_TIMEOUT;
+    }
+    return I8_OK;
+}
+
+int i8ops_last_cuda_error(void) { return t_last_cuda; }
+int i8ops_last_path(void) { return t_last_path; }
+
+int i8ops_set_path(int mode) {
+    const int prev = g_path_mode;
+    if (mode >= 0 && mode <= 2) g_path_mode = mode;
+    return prev;
+}
+
+void i8ops_set_wait_limit_ms(int ms) {
+    if (ms < 1) ms = 1;
+    g_wait_limit_ns = (uint64_t)ms * 1000ull * 1000ull;
+}
+
+int i8ops_version(void) { return 1; }
+
+}  // extern "C"

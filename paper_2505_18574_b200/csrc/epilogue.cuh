@@ -1,0 +1,84 @@
+// Fused read-out epilogue: bias -> ReLU -> fixed-point scale (round half up) -> saturate to int8.
+//
+// Two evaluations of the same exact function:
+//   requant_wide()  the definition, in 64-bit arithmetic (used by the generic kernel);
+//   requant_fast()  the tensor paths' version: per output channel a clamp window [lo, hi] is prepared
+//                   once, so that after clamping t = acc + bias into it (a) the saturated result is
+//                   unchanged and (b) floor((t*mult + r) / 2^shift) fits in 32 bits, which leaves one
+//                   widening multiply-add and one funnel shift per output.
+#pragma once
+#include <stdint.h>
+
+namespace i8 {
+
+__device__ __forceinline__ int32_t requant_wide(int32_t acc, int32_t bias, int relu, int32_t mult, int32_t shift) {
+    long long t = (long long)acc + (long long)bias;
+    if (relu && t < 0) t = 0;
+    const long long r = shift >= 1 ? (1ll << (shift - 1)) : 0ll;
+    long long u = (t * (long long)mult + r) >> shift;   // arithmetic shift on device = floor
+    u = u > 127 ? 127 : u;
+    u = u < -128 ? -128 : u;
+    return (int32_t)u;
+}
+
+// Per-output-channel constants of requant_fast.
+struct ChanConst {
+    int32_t lo, hi;     // clamp window for t = acc + bias (ReLU folded into lo)
+    int32_t mult;       // multiplier (canonicalised, see below)
+    int32_t shift;      // 0..31
+    int32_t rnd;        // 2^(shift-1), or 0 for shift 0
+};
+
+// Why the window is exact.  Let b = bit length of |mult| and e = shift + 9 - b.
+//   * |t| >= 2^e and mult != 0 imply |t*mult| >= 2^e * 2^(b-1) = 2^(shift+8), so the scaled value is at
+//     least 255.5 in magnitude and saturates to the same side as for any larger |t|: clamping t to
+//     [-2^e, 2^e] keeps the output.  (mult == 0 gives 0 for every t.)
+//   * |t| <= 2^e implies |t*mult + r| < 2^(shift+9) + 2^shift, so the shifted value is below 2^10 in
+//     magnitude and its low 32 bits are the value itself.
+//   * e >= 31: no clamp is needed; then b <= shift - 22 and |t*mult| < 2^(shift+9) all the same.
+//   * e < 0 is raised to 0 (window [-1, 1]): |t| >= 1 still saturates, and |t*mult + r| <= 2^31 + 2^30
+//     shifted by shift >= 1 fits; for shift == 0 the value is t*mult itself, which fits unless
+//     mult == INT32_MIN and t == -1.  That single pair (mult = -2^31, shift = 0) is replaced by
+//     mult = -2^30: every non-zero t saturates to the same side with either multiplier.
+__device__ __forceinline__ ChanConst make_chan_const(int32_t mult, int32_t shift, int relu) {
+    ChanConst c;
+    if (mult == INT32_MIN && shift == 0) mult = -(1 << 30);
+    const uint32_t mag = mult < 0 ? (uint32_t)0 - (uint32_t)mult : (uint32_t)mult;
+    const int b = 32 - __clz(mag);
+    int e = shift + 9 - b;
+    if (e < 0) e = 0;
+    if (e >= 31) {
+        c.lo = INT32_MIN;
+        c.hi = INT32_MAX;
+    } else {
+        c.hi = 1 << e;
+        c.lo = -(1 << e);
+    }
+    if (relu && c.lo < 0) c.lo = 0;
+    c.mult = mult;
+    c.shift = shift;
+    c.rnd = shift >= 1 ? (1 << (shift - 1)) : 0;
+    return c;
+}
+
+// t = acc + bias already formed by the caller when convenient; this takes acc and bias separately.
+__device__ __forceinline__ int32_t requant_fast(int32_t acc, int32_t bias, int32_t lo, int32_t hi, int32_t mult,
+                                                int32_t shift, int32_t rnd) {
+    int32_t t = acc + bias;
+    t = max(t, lo);
+    t = min(t, hi);
+    const long long p = (long long)t * (long long)mult + (long long)(uint32_t)rnd;
+    const uint32_t plo = (uint32_t)p, phi = (uint32_t)((unsigned long long)p >> 32);
+    return (int32_t)__funnelshift_r(plo, phi, (uint32_t)shift);   // low word of p >> shift, shift in 0..31
+}
+
+// Saturate four 32-bit values to int8 and pack them, v0 in the lowest byte.
+__device__ __forceinline__ uint32_t pack_sat4(int32_t v0, int32_t v1, int32_t v2, int32_t v3) {
+    v0 = min(max(v0, -128), 127);
+    v1 = min(max(v1, -128), 127);
+    v2 = min(max(v2, -128), 127);
+    v3 = min(max(v3, -128), 127);
+    return ((uint32_t)v0 & 0xffu) | (((uint32_t)v1 & 0xffu) << 8) | (((uint32_t)v2 & 0xffu) << 16) | ((uint32_t)v3 << 24);
+}
+
+}  // namespace i8

@@ -1,0 +1,274 @@
+// Large-tile tensor path: persistent, warp-specialised int8 GEMM for sm_100a.
+//
+//   warp 0      producer : TMA loads of a 128 x 128-byte A tile and a BN x 128-byte B tile per ring slot
+//   warp 1      MMA      : one thread issues tcgen05.mma kind::i8 (128 x BN x 32 per instruction) into one of two
+//                          tensor-memory accumulators; the first instruction of a tile overwrites, the rest accumulate
+//   warps 2..5  epilogue : read a finished accumulator (tcgen05.ld), apply bias/ReLU/scale/saturate, store int8
+//
+// The roles map onto the decoupled load / execute / store controllers of the accelerator that the paper
+// targets (Gemmini ISA description, Prompts appendix), and the two accumulators are the paper's
+// accumulator double-buffering (Code Examples appendix, the optimised 12544x64x256 GEMM), so that the
+// read-out of one tile overlaps the products of the next.
+#pragma once
+#include "epilogue.cuh"
+#include "ptx.cuh"
+
+namespace i8 {
+
+constexpr int BM = 128;          // rows per tile = tensor-memory lanes
+constexpr int BK = 128;          // bytes of K per ring slot = one 128-byte swizzle row
+constexpr int UMMA_K = 32;       // K per tcgen05.mma for 8-bit operands
+constexpr int TC_THREADS = 192;
+constexpr int EPI_THREADS = 128;
+
+struct TileSched {
+    int m_tiles, n_tiles, num_tiles, group_m;
+    __device__ __forceinline__ void map(int tile, int& m_blk, int& n_blk) const {
+        const int width = group_m * n_tiles;
+        const int g = tile / width;
+        const int first_m = g * group_m;
+        const int gsz = min(m_tiles - first_m, group_m);
+        const int local = tile - g * width;
+        m_blk = first_m + local % gsz;
+        n_blk = local / gsz;
+    }
+};
+
+struct GemmTcParams {
+    int8_t* C;
+    int64_t ldc;
+    const int32_t* bias;
+    const int32_t* mult;
+    const int32_t* shift;
+    int per_channel, relu;
+    int M, N, K;
+    int c_vec_ok;               // C and ldc are 16-byte aligned: full chunks go out as 16-byte stores
+    TileSched sched;
+    uint64_t wait_limit_ns;
+    unsigned* dev_status;
+};
+
+template <int BN, int STAGES>
+struct TcSmem {
+    static constexpr int A_BYTES = BM * BK;
+    static constexpr int B_BYTES = BN * BK;
+    static constexpr int OFF_A = 0;
+    static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
+    static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // 6 int32 arrays of BN entries
+    static constexpr int OFF_BAR = OFF_CONST + 6 * BN * 4;           // full[S], empty[S], acc_full[2], acc_empty[2]
+    static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 4) * 8;  // tensor-memory base, stop flag
+    static constexpr int TOTAL = OFF_MISC + 16;
+    static constexpr int DYN_BYTES = TOTAL + 1024;                   // slack to align the base to 1024 bytes
+    static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // BN in {64,128,256}: a power of two
+};
+
+// Epilogue arithmetic for one 32-column chunk held in v[]; column constants come from shared memory.
+__device__ __forceinline__ void epilogue_chunk(const int32_t (&v)[32], const int32_t* s_bias, const int32_t* s_lo,
+                                               const int32_t* s_hi, const int32_t* s_mult, const int32_t* s_shift,
+                                               const int32_t* s_rnd, int c0, uint32_t (&out)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+        const int4 bi = *reinterpret_cast<const int4*>(s_bias + c0 + 4 * j);
+        const int4 lo = *reinterpret_cast<const int4*>(s_lo + c0 + 4 * j);
+        const int4 hi = *reinterpret_cast<const int4*>(s_hi + c0 + 4 * j);
+        const int4 mu = *reinterpret_cast<const int4*>(s_mult + c0 + 4 * j);
+        const int4 sh = *reinterpret_cast<const int4*>(s_shift + c0 + 4 * j);
+        const int4 rn = *reinterpret_cast<const int4*>(s_rnd + c0 + 4 * j);
+        const int32_t r0 = requant_fast(v[4 * j + 0], bi.x, lo.x, hi.x, mu.x, sh.x, rn.x);
+        const int32_t r1 = requant_fast(v[4 * j + 1], bi.y, lo.y, hi.y, mu.y, sh.y, rn.y);
+        const int32_t r2 = requant_fast(v[4 * j + 2], bi.z, lo.z, hi.z, mu.z, sh.z, rn.z);
+        const int32_t r3 = requant_fast(v[4 * j + 3], bi.w, lo.w, hi.w, mu.w, sh.w, rn.w);
+        out[j] = pack_sat4(r0, r1, r2, r3);
+    }
+}
+
+// Store one thread's 32 output bytes (columns n .. n+31 of one row).
+__device__ __forceinline__ void store_row_chunk(int8_t* crow, int n, int N, bool vec_ok, const uint32_t (&out)[8]) {
+    if (vec_ok && n + 32 <= N) {
+        uint4* dst = reinterpret_cast<uint4*>(crow + n);
+        dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+        dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; j++)
+            if (n + j < N) crow[n + j] = (int8_t)((out[j >> 2] >> (8 * (j & 3))) & 0xff);
+    }
+}
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmTcParams p) {
+    using L = TcSmem<BN, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
+    uint8_t* smem = smem_raw + pad;
+    const uint32_t sbase = raw + pad;
+
+    const uint32_t sA = sbase + L::OFF_A, sB = sbase + L::OFF_B;
+    int32_t* s_bias = reinterpret_cast<int32_t*>(smem + L::OFF_CONST);
+    int32_t* s_lo = s_bias + BN;
+    int32_t* s_hi = s_lo + BN;
+    int32_t* s_mult = s_hi + BN;
+    int32_t* s_shift = s_mult + BN;
+    int32_t* s_rnd = s_shift + BN;
+    const uint32_t bar_full = sbase + L::OFF_BAR;
+    const uint32_t bar_empty = bar_full + STAGES * 8;
+    const uint32_t bar_acc_full = bar_empty + STAGES * 8;
+    const uint32_t bar_acc_empty = bar_acc_full + 2 * 8;
+    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC);
+    volatile int* s_stop = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const WaitEnv env{s_stop, p.dev_status, p.wait_limit_ns};
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; s++) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; b++) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, EPI_THREADS);
+        }
+        *s_stop = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(s_tmem)), L::TMEM_COLS);
+        tmem_relinquish();
+    }
+    if (warp == 0 && lane == 0) {
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *s_tmem;
+
+    const int num_kb = (p.K + BK - 1) / BK;
+    const TileSched sched = p.sched;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0, issued = 0, issued_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
+                int m_blk, n_blk;
+                sched.map(tile, m_blk, n_blk);
+                for (int kb = 0; kb < num_kb; kb++) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                    mbar_expect_tx(bar_full + 8 * stage, L::A_BYTES + L::B_BYTES);
+                    tma_load_2d(sA + stage * L::A_BYTES, &tmA, bar_full + 8 * stage, kb * BK, m_blk * BM);
+                    tma_load_2d(sB + stage * L::B_BYTES, &tmB, bar_full + 8 * stage, kb * BK, n_blk * BN);
+                    issued |= 1u << stage;
+                    issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+            if (*s_stop) {
+                // stopping early: let every copy this thread started land before the CTA retires
+                for (int s = 0; s < STAGES; s++)
+                    if (issued & (1u << s))
+                        if (!mbar_wait_drain(bar_full + 8 * s, (issued_phase >> s) & 1u, p.wait_limit_ns))
+                            atomicCAS(p.dev_status, 0u, (unsigned)DEV_TIMEOUT_DRAIN);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_i8(BM, BN, 0, 0);
+            int stage = 0, ab = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
+                if (!mbar_wait(bar_acc_empty + 8 * ab, acc_phase ^ 1, env, DEV_TIMEOUT_MMA_ACC)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + ab * BN;
+                for (int kb = 0; kb < num_kb; kb++) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, env, DEV_TIMEOUT_MMA_FULL)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a0 = sA + stage * L::A_BYTES, b0 = sB + stage * L::B_BYTES;
+                    const int rem = p.K - kb * BK;
+                    const int ksteps = rem >= BK ? BK / UMMA_K : (rem + UMMA_K - 1) / UMMA_K;
+                    for (int k = 0; k < ksteps; k++) {
+                        // K-major, 128-byte swizzle: rows 128 bytes apart, 8-row groups 1024 bytes apart;
+                        // a 32-byte step along K inside the swizzle row is a plain address offset.
+                        const uint64_t ad = make_smem_desc(a0 + k * UMMA_K, 16, 1024, SWZ_128B);
+                        const uint64_t bd = make_smem_desc(b0 + k * UMMA_K, 16, 1024, SWZ_128B);
+                        mma_i8_ss(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(bar_empty + 8 * stage);   // slot reusable once these MMAs have read it
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                tc_commit(bar_acc_full + 8 * ab);       // accumulator complete
+                ab ^= 1;
+                if (ab == 0) acc_phase ^= 1;
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue (4 warps = 128 lanes)
+        const int etid = threadIdx.x - 64;
+        const int quarter = warp & 3;                   // a warp may only read lanes 32*(warp%4) .. +31
+        int ab = 0, cached_n_blk = -1;
+        uint32_t acc_phase = 0;
+        for (int tile = blockIdx.x; tile < sched.num_tiles; tile += gridDim.x) {
+            int m_blk, n_blk;
+            sched.map(tile, m_blk, n_blk);
+            bool ok = mbar_wait(bar_acc_full + 8 * ab, acc_phase, env, DEV_TIMEOUT_EPILOGUE);
+            ok = named_barrier_and(1, EPI_THREADS, ok);   // all agree; also: previous tile's constants are no longer read
+            if (!ok) break;
+            tc_fence_after();
+            const int n0 = n_blk * BN;
+            if (n_blk != cached_n_blk) {
+                for (int c = etid; c < BN; c += EPI_THREADS) {
+                    const int n = n0 + c;
+                    int32_t bias = 0, mult = 0, shift = 0;
+                    if (n < p.N) {
+                        bias = p.bias ? p.bias[n] : 0;
+                        mult = p.mult[p.per_channel ? n : 0];
+                        shift = p.shift[p.per_channel ? n : 0];
+                    }
+                    const ChanConst cc = make_chan_const(mult, shift, p.relu);
+                    s_bias[c] = bias; s_lo[c] = cc.lo; s_hi[c] = cc.hi;
+                    s_mult[c] = cc.mult; s_shift[c] = cc.shift; s_rnd[c] = cc.rnd;
+                }
+                cached_n_blk = n_blk;
+                named_barrier(2, EPI_THREADS);
+            }
+            const int row = m_blk * BM + quarter * 32 + lane;
+            int8_t* crow = p.C + (int64_t)row * p.ldc;
+            const uint32_t t0 = tmem_base + ab * BN + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+            for (int ch = 0; ch < BN / 32; ch++) {
+                const int n = n0 + ch * 32;
+                if (n >= p.N) break;
+                int32_t v[32];
+                tmem_ld_32x32(t0 + ch * 32, v);
+                tmem_ld_wait();
+                uint32_t out[8];
+                epilogue_chunk(v, s_bias, s_lo, s_hi, s_mult, s_shift, s_rnd, ch * 32, out);
+                if (row < p.M) store_row_chunk(crow, n, p.N, p.c_vec_ok != 0, out);
+            }
+            tc_fence_before();
+            mbar_arrive(bar_acc_empty + 8 * ab);
+            ab ^= 1;
+            if (ab == 0) acc_phase ^= 1;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, L::TMEM_COLS);
+    }
+}
+
+}  // namespace i8

@@ -1,0 +1,68 @@
+// Generic kernels: one thread per output element, plain loops, any strides and alignments.
+// They serve operands the tensor paths cannot take (misaligned, MN-contiguous in unsupported
+// combinations, K == 0) and tiny problems, and double as an in-library cross-check of the tensor paths.
+#pragma once
+#include "epilogue.cuh"
+
+namespace i8 {
+
+struct GenericGemmParams {
+    const int8_t* A; int64_t a_rs, a_cs, a_bs;
+    const int8_t* B; int64_t b_rs, b_cs, b_bs;
+    int8_t* C; int64_t ldc, c_bs;
+    const int32_t* bias; int64_t bias_bs;
+    const int32_t* mult; const int32_t* shift;
+    int per_channel, relu;
+    int batch, M, N, K;
+};
+
+__global__ void __launch_bounds__(256) gemm_i8_generic_kernel(const GenericGemmParams p) {
+    const int64_t total = (int64_t)p.batch * p.M * p.N;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int n = (int)(idx % p.N);
+        const int64_t rest = idx / p.N;
+        const int m = (int)(rest % p.M);
+        const int64_t b = rest / p.M;
+        const int8_t* a = p.A + b * p.a_bs + (int64_t)m * p.a_rs;
+        const int8_t* bb = p.B + b * p.b_bs + (int64_t)n * p.b_cs;
+        int32_t acc = 0;
+        for (int k = 0; k < p.K; k++) acc += (int32_t)a[(int64_t)k * p.a_cs] * (int32_t)bb[(int64_t)k * p.b_rs];
+        const int32_t bias = p.bias ? p.bias[b * p.bias_bs + n] : 0;
+        const int ci = p.per_channel ? n : 0;
+        p.C[b * p.c_bs + (int64_t)m * p.ldc + n] = (int8_t)requant_wide(acc, bias, p.relu, p.mult[ci], p.shift[ci]);
+    }
+}
+
+struct GenericConvParams {
+    const int8_t* x; const int8_t* w; int8_t* y;
+    const int32_t* bias; const int32_t* mult; const int32_t* shift;
+    int per_channel, relu;
+    int N, H, W, C, K, R, S, P, Q, stride_h, stride_w, pad_h, pad_w;
+};
+
+__global__ void __launch_bounds__(256) conv2d_i8_generic_kernel(const GenericConvParams p) {
+    const int64_t total = (int64_t)p.N * p.P * p.Q * p.K;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int k = (int)(idx % p.K);
+        int64_t rest = idx / p.K;
+        const int q = (int)(rest % p.Q); rest /= p.Q;
+        const int pp = (int)(rest % p.P);
+        const int n = (int)(rest / p.P);
+        int32_t acc = 0;
+        for (int r = 0; r < p.R; r++) {
+            const int h = pp * p.stride_h - p.pad_h + r;
+            if (h < 0 || h >= p.H) continue;
+            for (int s = 0; s < p.S; s++) {
+                const int ww = q * p.stride_w - p.pad_w + s;
+                if (ww < 0 || ww >= p.W) continue;
+                const int8_t* xp = p.x + (((int64_t)n * p.H + h) * p.W + ww) * p.C;
+                const int8_t* wp = p.w + (((int64_t)k * p.R + r) * p.S + s) * p.C;
+                for (int c = 0; c < p.C; c++) acc += (int32_t)xp[c] * (int32_t)wp[c];
+            }
+        }
+        const int ci = p.per_channel ? k : 0;
+        p.y[idx] = (int8_t)requant_wide(acc, p.bias ? p.bias[k] : 0, p.relu, p.mult[ci], p.shift[ci]);
+    }
+}
+
+}  // namespace i8

@@ -1,0 +1,136 @@
+"""GPU parity: gemm_i8 through the C ABI against the CPU oracle, bit-exact."""
+import numpy as np
+import pytest
+
+from paper_2505_18574_b200 import inputs
+import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _auto_path():
+    import paper_2505_18574_b200 as i8
+    i8.set_path(0)
+    yield
+    i8.set_path(0)
+
+
+def _both_paths(p, expect_tensor=True):
+    import paper_2505_18574_b200 as i8
+    want = H.gemm_oracle(p)
+    i8.set_path(0)
+    got = H.gemm_gpu(p)
+    path = i8.last_path()
+    H.assert_same(got, want, f"{p.name} auto path={path}")
+    if expect_tensor:
+        assert path == i8.PATH_TENSOR, f"{p.name}: expected the tensor path, got {path}"
+    i8.set_path(1)
+    got = H.gemm_gpu(p)
+    assert i8.last_path() == i8.PATH_GENERIC
+    H.assert_same(got, want, f"{p.name} generic")
+    return want
+
+
+def test_config0_256cube():
+    want = _both_paths(inputs.config0())
+    H.not_degenerate(want)
+
+
+def test_single_tile_structured():
+    """Identity-like A and ramp B: a wrong descriptor field would show up as a recognisable permutation."""
+    M = N = K = 128
+    p = inputs.make_gemm(M, N, K, 1, per_channel=0, relu=0, with_bias=False)
+    p.A[:] = 0
+    for i in range(M):
+        p.A[i, i] = 1
+    for n in range(N):
+        for k in range(K):
+            p.B[n, k] = ((3 * k + 5 * n) % 251) - 125
+    p.mult[:] = 1; p.shift[:] = 0
+    want = _both_paths(p)
+    assert np.array_equal(want, p.B.T[:K, :N])     # I . B = B, no scaling
+
+
+@pytest.mark.parametrize("M,N,K", [
+    (128, 128, 128), (128, 256, 128), (128, 64, 32), (256, 512, 384), (1, 16, 16), (127, 65, 129),
+    (129, 257, 33), (300, 200, 100), (513, 96, 1040), (64, 700, 256), (1000, 40, 48), (5, 7, 16),
+    (130, 130, 2048), (384, 320, 16), (128, 8, 64),
+])
+def test_ragged_shapes(M, N, K):
+    # K is kept a multiple of 16 so the operands qualify for the tensor path (leading dimension rule)
+    p = inputs.make_gemm(M, N, K, 1000 + M + N + K, per_channel=1, relu=(M % 2), shift_lo=12, shift_hi=22)
+    _both_paths(p)
+
+
+@pytest.mark.parametrize("M,N,K,pads", [(200, 136, 96, (16, 32, 16)), (130, 70, 80, (48, 16, 3)), (64, 64, 64, (0, 0, 5))])
+def test_padded_leading_dimensions(M, N, K, pads):
+    p = inputs.make_gemm(M, N, K, 77, per_channel=1, relu=1, lda_pad=pads[0], ldb_pad=pads[1], ldc_pad=pads[2],
+                         shift_lo=12, shift_hi=20)
+    _both_paths(p)
+
+
+@pytest.mark.parametrize("a_layout,b_layout", [("row", "row"), ("col", "col"), ("col", "row")])
+def test_other_layouts_use_generic(a_layout, b_layout):
+    p = inputs.make_gemm(70, 50, 90, 5, a_layout=a_layout, b_layout=b_layout, per_channel=1, relu=0, shift_lo=10, shift_hi=18)
+    _both_paths(p, expect_tensor=False)
+
+
+def test_unaligned_k_falls_back():
+    p = inputs.make_gemm(65, 33, 37, 6, per_channel=0, relu=1, shared_shift=12)
+    _both_paths(p, expect_tensor=False)
+
+
+@pytest.mark.parametrize("mult,shift,relu", [(1, 0, 0), (-1, 0, 0), (2147483647, 31, 0), (-2147483648, 0, 0), (-2147483648, 31, 1),
+                                              (0, 5, 0), (3, 1, 1), (65536, 16, 0), (-20000, 20, 1), (1, 31, 0)])
+def test_extreme_scales(mult, shift, relu):
+    p = inputs.make_gemm(128, 96, 64, 9, per_channel=0, relu=relu)
+    p.mult[:] = mult; p.shift[:] = shift
+    _both_paths(p)
+
+
+def test_closed_forms_on_gpu():
+    """Oracle-independent: all-ones operands give K everywhere; extreme constants give 2^27 at K = 8192."""
+    import paper_2505_18574_b200 as i8
+    for (a, b, K, mult, shift, expect) in [(1, 1, 96, 1, 0, 96), (-128, -128, 8192, 1, 21, 64), (-128, 127, 8192, 1, 20, -127)]:
+        p = inputs.make_gemm(256, 128, K, 3, per_channel=0, relu=0, with_bias=False)
+        p.A[:] = a; p.B[:] = b; p.mult[:] = mult; p.shift[:] = shift
+        got = H.gemm_gpu(p)
+        assert i8.last_path() == i8.PATH_TENSOR
+        assert (got == expect).all(), (a, b, K, np.unique(got))
+
+
+def test_config1a_full():
+    p = inputs.config1(0)
+    import paper_2505_18574_b200 as i8
+    got = H.gemm_gpu(p)
+    assert i8.last_path() == i8.PATH_TENSOR
+    want = H.gemm_oracle(p)
+    H.assert_same(got, want, p.name)
+    H.not_degenerate(want)
+
+
+@pytest.mark.parametrize("j", [1, 2])
+def test_config1_large_sampled(j):
+    """Full-size launch, compared on 512 sampled rows (every column) the oracle computes one by one."""
+    import paper_2505_18574_b200 as i8
+    p = inputs.config1(j)
+    got = H.gemm_gpu(p)
+    assert i8.last_path() == i8.PATH_TENSOR
+    rng = np.random.default_rng(j)
+    rows = np.unique(np.concatenate([rng.integers(0, p.M, size=500), [0, 1, 127, 128, p.M - 129, p.M - 128, p.M - 1]]))
+    want = H.gemm_oracle_rows(p, rows)
+    H.assert_same(got[rows], want, p.name)
+    H.not_degenerate(want)
+    # cheap whole-output properties: per-channel saturation pattern must match the sampled rows' statistics
+    assert got.min() >= -128 and got.max() <= 127
+
+
+def test_config4a_tall_skinny():
+    import paper_2505_18574_b200 as i8
+    p = inputs.config4a()
+    got = H.gemm_gpu(p)
+    assert i8.last_path() in (i8.PATH_TENSOR, i8.PATH_SMALL)
+    want = H.gemm_oracle(p)
+    H.assert_same(got, want, p.name)
+    H.not_degenerate(want)
