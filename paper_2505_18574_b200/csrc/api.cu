@@ -41,6 +41,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 static EncodeTiledFn g_encode_tiled = nullptr;
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+static EncodeIm2colFn g_encode_im2col = nullptr;
 
 static int cuda_fail(cudaError_t e) {
     t_last_cuda = (int)e;
@@ -69,6 +74,10 @@ static int get_ctx(DeviceCtx** out) {
             CUDA_TRY(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &q));
             if (q != cudaDriverEntryPointSuccess || !fn) return cuda_fail(cudaErrorNotSupported);
             g_encode_tiled = (EncodeTiledFn)fn;
+            fn = nullptr;
+            CUDA_TRY(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeIm2col", &fn, 12000, cudaEnableDefault, &q));
+            if (q != cudaDriverEntryPointSuccess || !fn) return cuda_fail(cudaErrorNotSupported);
+            g_encode_im2col = (EncodeIm2colFn)fn;
         }
         const char* bn = getenv("I8OPS_FORCE_BN");
         if (bn) g_force_bn = atoi(bn);
@@ -95,17 +104,21 @@ static int make_tmap(CUtensorMap* tm, const void* base, int rank, const uint64_t
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ------------------------------------------------------------------------------------------------ launches
-template <int BN, int STAGES>
+static CUtensorMapSwizzle swizzle_for(int cb) {
+    return cb == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (cb == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+
+template <int BN, int STAGES, bool CONV, int EPI_WARPS>
 static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUtensorMap& tmB, GemmTcParams& p,
                      cudaStream_t st) {
     using L = TcSmem<BN, STAGES>;
-    auto kern = gemm_i8_tc_kernel<BN, STAGES>;
+    auto kern = gemm_i8_tc_kernel<BN, STAGES, CONV, EPI_WARPS>;
     if (!ctx->attr_set[slot]) {
         CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES));
         ctx->attr_set[slot] = true;
     }
     const int grid = p.sched.num_tiles < ctx->sm_count ? p.sched.num_tiles : ctx->sm_count;
-    kern<<<grid, TC_THREADS, L::DYN_BYTES, st>>>(tmA, tmB, p);
+    kern<<<grid, 64 + 32 * EPI_WARPS, L::DYN_BYTES, st>>>(tmA, tmB, p);
     CUDA_TRY(cudaGetLastError());
     return I8_OK;
 }
@@ -129,23 +142,17 @@ static int choose_bn(int M, int N, int sm_count) {
     return best;
 }
 
-static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
-                       const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
-                       int K, int relu, cudaStream_t st) {
-    const int bn = choose_bn(M, N, ctx->sm_count);
-    CUtensorMap tmA, tmB;
-    {
-        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
-        const uint64_t str[1] = {(uint64_t)lda};
-        const uint32_t box[2] = {BK, BM};
-        int rc = make_tmap(&tmA, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
-        if (rc) return rc;
-    }
+// Common tail of the tensor paths: B's tensor map (an N x K matrix with K contiguous), the tile schedule,
+// and the launch of the instance that matches the tile width.
+static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop& kl, int bn, const int8_t* B, int64_t ldb,
+                  int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
+                  int M, int N, int K, int relu, cudaStream_t st) {
+    CUtensorMap tmB;
     {
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
         const uint64_t str[1] = {(uint64_t)ldb};
-        const uint32_t box[2] = {BK, (uint32_t)bn};
-        int rc = make_tmap(&tmB, B, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+        const uint32_t box[2] = {(uint32_t)kl.cb, (uint32_t)bn};
+        int rc = make_tmap(&tmB, B, 2, dims, str, box, swizzle_for(kl.cb));
         if (rc) return rc;
     }
     GemmTcParams p;
@@ -156,13 +163,63 @@ static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_
     p.sched.n_tiles = (N + bn - 1) / bn;
     p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
     p.sched.group_m = 16;
+    p.kl = kl;
     p.wait_limit_ns = g_wait_limit_ns;
     p.dev_status = ctx->dev_status;
-    switch (bn) {
-        case 256: return launch_tc<256, 4>(ctx, 0, tmA, tmB, p, st);
-        case 128: return launch_tc<128, 6>(ctx, 1, tmA, tmB, p, st);
-        default:  return launch_tc<64, 8>(ctx, 2, tmA, tmB, p, st);
+    if (conv) {
+        switch (bn) {
+            case 256: return launch_tc<256, 4, true, 8>(ctx, 3, tmA, tmB, p, st);
+            case 128: return launch_tc<128, 6, true, 8>(ctx, 4, tmA, tmB, p, st);
+            default:  return launch_tc<64, 8, true, 8>(ctx, 5, tmA, tmB, p, st);
+        }
     }
+    switch (bn) {
+        case 256: return launch_tc<256, 4, false, 4>(ctx, 0, tmA, tmB, p, st);
+        case 128: return launch_tc<128, 6, false, 4>(ctx, 1, tmA, tmB, p, st);
+        default:  return launch_tc<64, 8, false, 8>(ctx, 2, tmA, tmB, p, st);
+    }
+}
+
+static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
+                       const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
+                       int K, int relu, cudaStream_t st) {
+    const int bn = choose_bn(M, N, ctx->sm_count);
+    CUtensorMap tmA;
+    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
+    const uint64_t str[1] = {(uint64_t)lda};
+    const uint32_t box[2] = {BK, BM};
+    int rc = make_tmap(&tmA, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    KLoop kl{};
+    kl.cb = BK; kl.nsub = 1; kl.num_kblocks = (K + BK - 1) / BK;
+    return run_tc(ctx, false, tmA, kl, bn, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
+}
+
+// Implicit-GEMM convolution: A tiles come from an im2col-mode tensor map over the NHWC activations.
+static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, const int32_t* mult,
+                       const int32_t* shift, int per_channel, int N, int H, int W, int C, int Kf, int R, int S, int P, int Q,
+                       int stride_h, int stride_w, int pad_h, int pad_w, int relu, cudaStream_t st) {
+    const int cb = C % 128 == 0 ? 128 : (C % 64 == 0 ? 64 : 32);
+    const int M = N * P * Q;
+    const int bn = choose_bn(M, Kf, ctx->sm_count);
+    CUtensorMap tmA;
+    {
+        const cuuint64_t gdim[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+        const cuuint64_t gstr[3] = {(cuuint64_t)C, (cuuint64_t)W * C, (cuuint64_t)H * W * C};
+        const int lower[2] = {-pad_w, -pad_h};
+        const int upper[2] = {pad_w - (S - 1), pad_h - (R - 1)};
+        const cuuint32_t estr[4] = {1, (cuuint32_t)stride_w, (cuuint32_t)stride_h, 1};
+        CUresult r = g_encode_im2col(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(x), gdim, gstr, lower, upper,
+                                     (cuuint32_t)cb, (cuuint32_t)BM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(cb),
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) { t_last_cuda = (int)cudaErrorInvalidValue; return I8_ERR_CUDA; }
+    }
+    KLoop kl{};
+    kl.cb = cb; kl.nsub = BK / cb; kl.cblocks = C / cb; kl.num_kblocks = R * S * kl.cblocks;
+    kl.P = P; kl.Q = Q; kl.S = S;
+    kl.stride_h = stride_h; kl.stride_w = stride_w; kl.pad_h = pad_h; kl.pad_w = pad_w;
+    const int K = R * S * C;
+    return run_tc(ctx, true, tmA, kl, bn, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
 }
 
 static int run_gemm_generic(const GenericGemmParams& p, cudaStream_t st) {
@@ -260,6 +317,24 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
     int rc = get_ctx(&ctx);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    if (g_path_mode != 1 && aligned16(x) && aligned16(w)) {
+        if (R == 1 && S == 1 && stride_h == 1 && stride_w == 1 && pad_h == 0 && pad_w == 0 && C % 16 == 0) {
+            // a 1x1 convolution is the GEMM [N*H*W, C] x [C, K]
+            rc = run_gemm_tc(ctx, x, C, w, C, y, K, bias, mult, shift, per_channel, N * H * W, K, C, relu, st);
+            if (rc == I8_OK) t_last_path = I8_PATH_TENSOR;
+            return rc;
+        }
+        // im2col tensor maps: channel blocks of 32/64/128 bytes, box corners and tap offsets within the 4-D
+        // encoding's ranges, traversal strides up to 8; activation tensors below 128 KiB stay on the generic kernel
+        const bool tc_legal = C % 32 == 0 && R <= 16 && S <= 16 && pad_h <= 16 && pad_w <= 16 && stride_h <= 8 &&
+                              stride_w <= 8 && (int64_t)N * H * W * C >= 131072 && (int64_t)N * P * Q < (1ll << 31);
+        if (tc_legal) {
+            rc = run_conv_tc(ctx, x, w, y, bias, mult, shift, per_channel, N, H, W, C, K, R, S, P, Q, stride_h, stride_w,
+                             pad_h, pad_w, relu, st);
+            if (rc == I8_OK) t_last_path = I8_PATH_TENSOR;
+            return rc;
+        }
+    }
     GenericConvParams g{x, w, y, bias, mult, shift, per_channel, relu, N, H, W, C, K, R, S, P, Q, stride_h, stride_w, pad_h, pad_w};
     const int64_t total = (int64_t)N * P * Q * K;
     int64_t blocks = (total + 255) / 256;

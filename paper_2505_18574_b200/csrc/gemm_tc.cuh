@@ -3,7 +3,14 @@
 //   warp 0      producer : TMA loads of a 128 x 128-byte A tile and a BN x 128-byte B tile per ring slot
 //   warp 1      MMA      : one thread issues tcgen05.mma kind::i8 (128 x BN x 32 per instruction) into one of two
 //                          tensor-memory accumulators; the first instruction of a tile overwrites, the rest accumulate
-//   warps 2..5  epilogue : read a finished accumulator (tcgen05.ld), apply bias/ReLU/scale/saturate, store int8
+//   warps 2..   epilogue : 4 or 8 warps read a finished accumulator (tcgen05.ld), apply bias/ReLU/scale/saturate,
+//                          store int8
+//
+// The same kernel serves the convolution as an implicit GEMM (M = N*P*Q output pixels, N = filters,
+// K = R*S*C): there the producer fetches A with TMA im2col loads straight from the NHWC activations, one
+// load per filter tap and channel block, padding supplied by the out-of-bounds zero fill; no im2col
+// matrix ever exists in memory.  A ring slot always holds 128 bytes of K per row, as 1, 2 or 4 sub-blocks
+// of cb = 128, 64 or 32 bytes (cb = the channel block; plain GEMMs use one 128-byte block).
 //
 // The roles map onto the decoupled load / execute / store controllers of the accelerator that the paper
 // targets (Gemmini ISA description, Prompts appendix), and the two accumulators are the paper's
@@ -18,8 +25,14 @@ namespace i8 {
 constexpr int BM = 128;          // rows per tile = tensor-memory lanes
 constexpr int BK = 128;          // bytes of K per ring slot = one 128-byte swizzle row
 constexpr int UMMA_K = 32;       // K per tcgen05.mma for 8-bit operands
-constexpr int TC_THREADS = 192;
-constexpr int EPI_THREADS = 128;
+
+// Geometry of the K loop.  GEMM: cb = 128, nsub = 1, num_kblocks = ceil(K / 128).
+// Convolution: cb = channel block, nsub = 128 / cb, num_kblocks = R * S * (C / cb).
+struct KLoop {
+    int cb, nsub, num_kblocks;
+    int P, Q, S, cblocks;                 // convolution only: output extent, filter width, C / cb
+    int stride_h, stride_w, pad_h, pad_w;
+};
 
 struct TileSched {
     int m_tiles, n_tiles, num_tiles, group_m;
@@ -44,6 +57,7 @@ struct GemmTcParams {
     int M, N, K;
     int c_vec_ok;               // C and ldc are 16-byte aligned: full chunks go out as 16-byte stores
     TileSched sched;
+    KLoop kl;
     uint64_t wait_limit_ns;
     unsigned* dev_status;
 };
@@ -95,10 +109,16 @@ __device__ __forceinline__ void store_row_chunk(int8_t* crow, int n, int N, bool
     }
 }
 
-template <int BN, int STAGES>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+template <int BN, int STAGES, bool CONV, int EPI_WARPS>
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmTcParams p) {
     using L = TcSmem<BN, STAGES>;
+    constexpr int EPI_THREADS = 32 * EPI_WARPS;
+    constexpr int COL_GROUPS = EPI_WARPS / 4;          // warps sharing a lane quarter split the columns
+    constexpr int COLS_PER_GROUP = BN / COL_GROUPS;
+    static_assert(EPI_WARPS == 4 || EPI_WARPS == 8, "4 or 8 epilogue warps");
+    static_assert(COLS_PER_GROUP % 32 == 0, "column split must keep 32-column chunks");
+
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -147,8 +167,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *s_tmem;
 
-    const int num_kb = (p.K + BK - 1) / BK;
     const TileSched sched = p.sched;
+    const KLoop kl = p.kl;
+    const uint32_t a_sub_bytes = BM * kl.cb, b_sub_bytes = BN * kl.cb;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -159,11 +180,34 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
                 int m_blk, n_blk;
                 sched.map(tile, m_blk, n_blk);
-                for (int kb = 0; kb < num_kb; kb++) {
+                int w0 = 0, h0 = 0, img = 0;
+                if (CONV) {
+                    // first output pixel of the tile -> position of filter tap (0,0) in the input image
+                    const int m0 = m_blk * BM;
+                    const int pq = kl.P * kl.Q;
+                    img = m0 / pq;
+                    const int rem = m0 - img * pq;
+                    const int op = rem / kl.Q, oq = rem - op * kl.Q;
+                    h0 = op * kl.stride_h - kl.pad_h;
+                    w0 = oq * kl.stride_w - kl.pad_w;
+                }
+                int c_idx = 0, fs = 0, fr = 0;      // convolution: channel block, filter column, filter row
+                for (int kbi = 0; kbi < kl.num_kblocks;) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
-                    mbar_expect_tx(bar_full + 8 * stage, L::A_BYTES + L::B_BYTES);
-                    tma_load_2d(sA + stage * L::A_BYTES, &tmA, bar_full + 8 * stage, kb * BK, m_blk * BM);
-                    tma_load_2d(sB + stage * L::B_BYTES, &tmB, bar_full + 8 * stage, kb * BK, n_blk * BN);
+                    const int nb = min(kl.nsub, kl.num_kblocks - kbi);
+                    const uint32_t full = bar_full + 8 * stage;
+                    mbar_expect_tx(full, nb * (a_sub_bytes + b_sub_bytes));
+                    for (int j = 0; j < nb; j++, kbi++) {
+                        const uint32_t dstA = sA + stage * L::A_BYTES + j * a_sub_bytes;
+                        const uint32_t dstB = sB + stage * L::B_BYTES + j * b_sub_bytes;
+                        if (CONV) {
+                            tma_load_im2col_4d(dstA, &tmA, full, c_idx * kl.cb, w0, h0, img, (uint16_t)fs, (uint16_t)fr);
+                            if (++c_idx == kl.cblocks) { c_idx = 0; if (++fs == kl.S) { fs = 0; ++fr; } }
+                        } else {
+                            tma_load_2d(dstA, &tmA, full, kbi * BK, m_blk * BM);
+                        }
+                        tma_load_2d(dstB, &tmB, full, kbi * kl.cb, n_blk * BN);
+                    }
                     issued |= 1u << stage;
                     issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -182,6 +226,10 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_i8(BM, BN, 0, 0);
+            // K-major operands: rows cb bytes apart, swizzled over cb bytes, 8-row groups 8*cb bytes apart;
+            // a 32-byte step along K inside a swizzle row is a plain address offset.
+            const uint64_t swz = kl.cb == 128 ? SWZ_128B : (kl.cb == 64 ? SWZ_64B : SWZ_32B);
+            const uint32_t sbo = 8 * kl.cb;
             int stage = 0, ab = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
@@ -189,18 +237,25 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 if (!mbar_wait(bar_acc_empty + 8 * ab, acc_phase ^ 1, env, DEV_TIMEOUT_MMA_ACC)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + ab * BN;
-                for (int kb = 0; kb < num_kb; kb++) {
+                uint32_t accumulate = 0;
+                for (int kbi = 0; kbi < kl.num_kblocks;) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, env, DEV_TIMEOUT_MMA_FULL)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a0 = sA + stage * L::A_BYTES, b0 = sB + stage * L::B_BYTES;
-                    const int rem = p.K - kb * BK;
-                    const int ksteps = rem >= BK ? BK / UMMA_K : (rem + UMMA_K - 1) / UMMA_K;
-                    for (int k = 0; k < ksteps; k++) {
-                        // K-major, 128-byte swizzle: rows 128 bytes apart, 8-row groups 1024 bytes apart;
-                        // a 32-byte step along K inside the swizzle row is a plain address offset.
-                        const uint64_t ad = make_smem_desc(a0 + k * UMMA_K, 16, 1024, SWZ_128B);
-                        const uint64_t bd = make_smem_desc(b0 + k * UMMA_K, 16, 1024, SWZ_128B);
-                        mma_i8_ss(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+                    const int nb = min(kl.nsub, kl.num_kblocks - kbi);
+                    for (int j = 0; j < nb; j++, kbi++) {
+                        const uint32_t a0 = sA + stage * L::A_BYTES + j * a_sub_bytes;
+                        const uint32_t b0 = sB + stage * L::B_BYTES + j * b_sub_bytes;
+                        int ksteps = kl.cb / UMMA_K;
+                        if (!CONV) {                       // GEMM: the last block may be ragged in K
+                            const int rem = p.K - kbi * BK;
+                            if (rem < BK) ksteps = (rem + UMMA_K - 1) / UMMA_K;
+                        }
+                        for (int k = 0; k < ksteps; k++) {
+                            const uint64_t ad = make_smem_desc(a0 + k * UMMA_K, 16, sbo, swz);
+                            const uint64_t bd = make_smem_desc(b0 + k * UMMA_K, 16, sbo, swz);
+                            mma_i8_ss(d_tmem, ad, bd, idesc, accumulate);
+                            accumulate = 1;
+                        }
                     }
                     tc_commit(bar_empty + 8 * stage);   // slot reusable once these MMAs have read it
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -213,9 +268,10 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ epilogue (4 warps = 128 lanes)
+        // ------------------------------------------------------------------ epilogue
         const int etid = threadIdx.x - 64;
         const int quarter = warp & 3;                   // a warp may only read lanes 32*(warp%4) .. +31
+        const int cgroup = (warp - 2) >> 2;             // which share of the columns this warp handles
         int ab = 0, cached_n_blk = -1;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < sched.num_tiles; tile += gridDim.x) {
@@ -246,14 +302,15 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             int8_t* crow = p.C + (int64_t)row * p.ldc;
             const uint32_t t0 = tmem_base + ab * BN + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
-            for (int ch = 0; ch < BN / 32; ch++) {
-                const int n = n0 + ch * 32;
+            for (int ch = 0; ch < COLS_PER_GROUP / 32; ch++) {
+                const int c0 = cgroup * COLS_PER_GROUP + ch * 32;
+                const int n = n0 + c0;
                 if (n >= p.N) break;
                 int32_t v[32];
-                tmem_ld_32x32(t0 + ch * 32, v);
+                tmem_ld_32x32(t0 + c0, v);
                 tmem_ld_wait();
                 uint32_t out[8];
-                epilogue_chunk(v, s_bias, s_lo, s_hi, s_mult, s_shift, s_rnd, ch * 32, out);
+                epilogue_chunk(v, s_bias, s_lo, s_hi, s_mult, s_shift, s_rnd, c0, out);
                 if (row < p.M) store_row_chunk(crow, n, p.N, p.c_vec_ok != 0, out);
             }
             tc_fence_before();

@@ -1,0 +1,123 @@
+"""GPU parity: conv2d_i8 and batched_gemm_i8 through the C ABI against the CPU oracle, bit-exact."""
+import numpy as np
+import pytest
+
+from paper_2505_18574_b200 import inputs
+import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _auto_path():
+    import paper_2505_18574_b200 as i8
+    i8.set_path(0)
+    yield
+    i8.set_path(0)
+
+
+def _conv_both(p, expect_tensor=None):
+    import paper_2505_18574_b200 as i8
+    want = H.conv_oracle(p)
+    i8.set_path(0)
+    got = H.conv_gpu(p)
+    path = i8.last_path()
+    H.assert_same(got, want, f"{p.name} auto path={path}")
+    if expect_tensor is not None:
+        assert (path == i8.PATH_TENSOR) == expect_tensor, f"{p.name}: path {path}"
+    i8.set_path(1)
+    got = H.conv_gpu(p)
+    assert i8.last_path() == i8.PATH_GENERIC
+    H.assert_same(got, want, f"{p.name} generic")
+    return want
+
+
+@pytest.mark.parametrize("N,H_,W,C,K,R,S,st,pad", [
+    (1, 8, 8, 64, 64, 3, 3, 1, 1), (2, 9, 7, 64, 32, 3, 3, 1, 1), (3, 12, 12, 128, 64, 3, 3, 2, 1),
+    (2, 7, 7, 256, 128, 1, 1, 1, 0), (1, 5, 5, 3, 4, 3, 3, 1, 1), (2, 10, 11, 16, 24, 5, 5, 2, 2),
+    (2, 14, 14, 64, 96, 3, 3, 1, 0), (1, 6, 6, 32, 16, 1, 1, 2, 0), (4, 28, 28, 64, 64, 3, 3, 1, 1),
+    (2, 15, 13, 192, 80, 3, 3, 2, 1), (1, 4, 4, 512, 64, 3, 3, 1, 1),
+])
+def test_conv_shapes(N, H_, W, C, K, R, S, st, pad):
+    p = inputs.make_conv(N, H_, W, C, K, R, S, st, pad, 300 + N + H_ + C + K)
+    _conv_both(p)
+
+
+@pytest.mark.parametrize("N,H_,W,C,K,R,S,st,pad", [
+    (4, 28, 28, 64, 64, 3, 3, 1, 1),      # 64-byte channel block, two taps per ring slot, odd tap count
+    (8, 12, 12, 128, 64, 3, 3, 2, 1),     # 128-byte channel block, stride 2
+    (4, 15, 13, 192, 80, 3, 3, 2, 1),     # 64-byte blocks x3, odd image, ragged filter count
+    (8, 24, 24, 32, 48, 3, 3, 1, 1),      # 32-byte channel block, four taps per slot
+    (4, 20, 22, 96, 40, 5, 5, 2, 2),      # 5x5 filter, 32-byte blocks x3
+    (6, 14, 14, 256, 256, 3, 3, 1, 1),    # two 128-byte blocks per tap
+    (5, 17, 17, 128, 136, 3, 3, 1, 0),    # no padding: the output is smaller than the input
+    (9, 16, 16, 64, 64, 1, 1, 2, 0),      # strided 1x1
+    (2, 40, 36, 64, 192, 3, 3, 1, 1),     # tiles spanning several rows and both images
+    (3, 30, 30, 64, 64, 7, 7, 2, 3),      # 7x7 stride 2 pad 3
+])
+def test_conv_tensor_path(N, H_, W, C, K, R, S, st, pad):
+    assert N * H_ * W * C >= 131072
+    p = inputs.make_conv(N, H_, W, C, K, R, S, st, pad, 500 + N + H_ + C + K)
+    _conv_both(p, expect_tensor=True)
+
+
+def test_conv_delta_filter_on_gpu():
+    """Oracle-independent: a filter with a single 1 copies a shifted view of the input."""
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_conv(24, 9, 10, 64, 64, 3, 3, 1, 1, 5, per_channel=0, relu=0, with_bias=False, act_lo=-100, act_hi=101)
+    p.mult[:] = 1; p.shift[:] = 0
+    for (r, s) in [(0, 0), (1, 1), (2, 0), (1, 2)]:
+        p.w[:] = 0
+        for k in range(64):
+            p.w[k, r, s, (k + 3) % 64] = 1
+        got = H.conv_gpu(p)
+        assert i8.last_path() == i8.PATH_TENSOR
+        for pp in range(p.P):
+            for q in range(p.Q):
+                h = pp - 1 + r; w = q - 1 + s
+                want = p.x[:, h, w, :][:, [(k + 3) % 64 for k in range(64)]] if (0 <= h < 9 and 0 <= w < 10) else 0
+                assert np.array_equal(got[:, pp, q, :], np.broadcast_to(want, (24, 64))), (r, s, pp, q)
+
+
+def test_conv_1x1_equals_gemm_on_gpu():
+    p = inputs.make_conv(3, 7, 7, 128, 256, 1, 1, 1, 0, 8)
+    y = H.conv_gpu(p)
+    g = inputs.make_gemm(3 * 49, 256, 128, 0, per_channel=1, relu=1)
+    g.A = p.x.reshape(-1, 128).copy(); g.B = p.w.reshape(256, 128).copy()
+    g.bias, g.mult, g.shift = p.bias, p.mult, p.shift
+    H.assert_same(y.reshape(-1, 256), H.gemm_gpu(g), "1x1 conv vs gemm")
+
+
+def test_config2_conv():
+    p = inputs.config2()
+    want = H.conv_oracle(p)
+    H.assert_same(H.conv_gpu(p), want, p.name)
+    H.not_degenerate(want)
+
+
+@pytest.mark.parametrize("j", [0, 1, 2])
+def test_config3_conv_mix(j):
+    p = inputs.config3(j)
+    want = H.conv_oracle(p)
+    H.assert_same(H.conv_gpu(p), want, p.name)
+    H.not_degenerate(want)
+
+
+@pytest.mark.parametrize("batch,M,N,K,ppb", [(1, 64, 64, 64, True), (7, 64, 64, 64, True), (8, 64, 64, 64, False),
+                                             (5, 32, 48, 80, True), (3, 128, 64, 64, True), (9, 17, 19, 23, True),
+                                             (33, 64, 64, 64, True)])
+def test_batched_shapes(batch, M, N, K, ppb):
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_batched(batch, M, N, K, 400 + batch + M, per_problem_bias=ppb)
+    p.shift[:] = 14
+    want = H.batched_oracle(p)
+    for mode in (0, 1):
+        i8.set_path(mode)
+        H.assert_same(H.batched_gpu(p), want, f"{p.name} mode {mode}")
+
+
+def test_config4b_batched():
+    p = inputs.config4b()
+    want = H.batched_oracle(p)
+    H.assert_same(H.batched_gpu(p), want, p.name)
+    H.not_degenerate(want)

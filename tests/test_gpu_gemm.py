@@ -58,8 +58,10 @@ def test_single_tile_structured():
     (130, 130, 2048), (384, 320, 16), (128, 8, 64),
 ])
 def test_ragged_shapes(M, N, K):
-    # K is kept a multiple of 16 so the operands qualify for the tensor path (leading dimension rule)
-    p = inputs.make_gemm(M, N, K, 1000 + M + N + K, per_channel=1, relu=(M % 2), shift_lo=12, shift_hi=22)
+    # leading dimensions are padded to a multiple of 16 so the operands qualify for the tensor path
+    pad = (-K) % 16
+    p = inputs.make_gemm(M, N, K, 1000 + M + N + K, per_channel=1, relu=(M % 2), shift_lo=12, shift_hi=22,
+                         lda_pad=pad, ldb_pad=pad)
     _both_paths(p)
 
 
