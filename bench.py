@@ -20,7 +20,6 @@ import statistics
 import subprocess
 import sys
 import tempfile
-import threading
 import time
 
 import numpy as np
@@ -57,53 +56,64 @@ def gemm_bytes(p):
 
 # ------------------------------------------------------------------------------------------------ clocks
 class ClockSampler:
-    """nvidia-smi sampled in the background during the timed region."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    """nvidia-smi sampled in the background; samples are attributed to the timed region by their timestamps."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
         self.gpu = gpu_index
         self.proc = None
-        self.tmp = None
+        self.path = None
 
     def start(self):
+        """Start sampling and wait (up to 5 s) for the first sample so the timed region is covered."""
         try:
-            self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                                          "-lms", "20", "-i", str(self.gpu)], stdout=open(self.path, "w"),
+                                         stderr=subprocess.DEVNULL)
+            t0 = time.time()
+            while time.time() - t0 < 5.0 and os.path.getsize(self.path) == 0:
+                time.sleep(0.02)
         except Exception:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, t_begin: float, t_end: float):
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "timed region"}
         if self.proc is None:
             return out
         try:
+            time.sleep(0.05)
             self.proc.terminate()
             self.proc.wait(timeout=5)
-        except Exception:
-            pass
-        try:
-            self.tmp.flush()
-            rows = [l.strip().split(", ") for l in open(self.tmp.name) if l.strip()]
-            os.unlink(self.tmp.name)
+            rows = [l.strip().split(", ") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
         except Exception:
             return out
-        sm, reasons, mx = [], set(), None
+        inside, anyload, mx = [], [], None
         for r in rows:
             if len(r) < 9:
                 continue
             try:
-                sm.append(float(r[1])); mx = float(r[2])
+                ts = datetime.datetime.strptime(r[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                mhz = float(r[1]); mx = float(r[2])
             except ValueError:
                 continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
-                if v.strip().lower().startswith("active"):
-                    reasons.add(name)
-        if sm:
-            busy = sorted(sm)[len(sm) // 4:]      # drop the idle quarter at the edges of the window
-            out.update(sm_mhz=statistics.median(busy), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+            reasons = [name for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9])
+                       if v.strip().lower().startswith("active")]
+            anyload.append((mhz, reasons))
+            if t_begin - 0.01 <= ts <= t_end + 0.01:
+                inside.append((mhz, reasons))
+        use = inside
+        if not use:
+            use = anyload
+            out["window"] = "whole run (timed region shorter than the sampling period)"
+        if use:
+            out.update(sm_mhz=statistics.median([u[0] for u in use]), sm_max_mhz=mx,
+                       reasons=sorted({x for u in use for x in u[1]}), samples=len(use))
         return out
 
 
@@ -166,7 +176,7 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -236,16 +246,17 @@ def main():
             got = dev_t[j]["C"][torch.from_numpy(rows).to(dev)].cpu().numpy()
             bit_exact = bit_exact and bool(np.array_equal(got, want))
 
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
     for _ in range(args.warmup):
         launch(0); launch(1); launch(2)
     barrier()
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     n_launch = 3 * args.steps
     evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_launch + 1)]
     barrier()
+    t_begin = time.time()
     evs[0].record()
     k = 0
     for _ in range(args.steps):
@@ -254,7 +265,8 @@ def main():
             k += 1
             evs[k].record()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    t_end = time.time()
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     total_ms = evs[0].elapsed_time(evs[-1])
     per_problem_ms = [0.0, 0.0, 0.0]
     for s in range(args.steps):
@@ -302,7 +314,8 @@ def main():
     details = None
     if args.details and rank == 0:
         from paper_2505_18574_b200 import bench_details
-        details = bench_details.run(dev)
+        pk = measured_peaks()
+        details = bench_details.run(dev, peak_tops=2 * pk["bf16_burst"], peak_gbs=pk["hbm_gbs"])
 
     if rank == 0:
         peaks = measured_peaks()
@@ -328,7 +341,7 @@ def main():
                     "steps": args.e2e_steps, "matches_device_path": bool(e2e_exact)},
             "gpu_launches": n_launch,
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                       "samples": clocks["samples"]},
+                       "samples": clocks["samples"], "window": clocks["window"]},
             "bit_exact_vs_oracle_sampled": bit_exact,
         }
         if cpu_baseline is not None:

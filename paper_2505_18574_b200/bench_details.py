@@ -1,0 +1,126 @@
+"""Per-problem timings of every workload configuration (GEMM 256^3, the three large GEMMs, the four
+convolutions, the tall-skinny GEMM and the batched 64^3 products) through the C-ABI binding.
+
+    python -m paper_2505_18574_b200.bench_details [--cfg 0,1a,2,...] [--iters N] [--no-graph]
+
+For each problem: device time per launch from back-to-back launches between two CUDA events, the same from
+a CUDA graph of the launches (launch gaps removed), int8 TOPS, algorithmic GB/s (every operand read once,
+the output written once) and the fraction of the roofline max(ops / tensor peak, bytes / HBM peak).
+Problems whose operands fit in L2 are rotated over enough copies of their buffers to exceed it.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+
+ALL = ["0", "1a", "1b", "1c", "2", "3a", "3b", "3c", "4a", "4b"]
+L2_BYTES = 126e6
+
+
+def _problem(name):
+    from . import inputs
+    return {"0": inputs.config0, "1a": lambda: inputs.config1(0), "1b": lambda: inputs.config1(1),
+            "1c": lambda: inputs.config1(2), "2": inputs.config2, "3a": lambda: inputs.config3(0),
+            "3b": lambda: inputs.config3(1), "3c": lambda: inputs.config3(2), "4a": inputs.config4a,
+            "4b": inputs.config4b}[name]()
+
+
+def _make(name, dev, copies_for_l2=True):
+    """Returns (launch(i), ops, algorithmic bytes, number of buffer sets)."""
+    import torch
+    from . import binding as i8
+    from . import inputs
+    p = _problem(name)
+
+    def T(a):
+        return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+
+    if isinstance(p, inputs.GemmProblem):
+        ops = 2.0 * p.M * p.N * p.K
+        byts = p.M * p.K + p.N * p.K + p.M * p.N + 4 * p.N + 8 * (p.N if p.per_channel else 1)
+        sets = int(min(16, max(1, np.ceil(2 * L2_BYTES / byts)))) if copies_for_l2 else 1
+        bufs = [(T(p.A), T(p.B), torch.empty((p.M, p.N), dtype=torch.int8, device=dev)) for _ in range(sets)]
+        b, mu, sh = T(p.bias), T(p.mult), T(p.shift)
+
+        def launch(i):
+            A, B, C = bufs[i % sets]
+            i8.gemm_i8(A, B.t(), C, b, mu, sh, p.per_channel, p.relu)
+    elif isinstance(p, inputs.ConvProblem):
+        ops = 2.0 * p.N * p.P * p.Q * p.K * p.R * p.S * p.C
+        byts = p.x.size + p.w.size + p.N * p.P * p.Q * p.K + 12 * p.K
+        sets = int(min(32, max(1, np.ceil(2 * L2_BYTES / byts)))) if copies_for_l2 else 1
+        bufs = [(T(p.x), T(p.w), torch.empty((p.N, p.P, p.Q, p.K), dtype=torch.int8, device=dev)) for _ in range(sets)]
+        b, mu, sh = T(p.bias), T(p.mult), T(p.shift)
+
+        def launch(i):
+            x, w, y = bufs[i % sets]
+            i8.conv2d_i8(x, w, y, b, mu, sh, p.per_channel, p.relu, (p.stride_h, p.stride_w), (p.pad_h, p.pad_w))
+    else:
+        ops = 2.0 * p.batch * p.M * p.N * p.K
+        byts = p.A.size + p.B.size + p.batch * p.M * p.N + p.bias.size * 4
+        sets = 1
+        A, B, C = T(p.A), T(p.B), torch.empty((p.batch, p.M, p.N), dtype=torch.int8, device=dev)
+        b, mu, sh = T(p.bias), T(p.mult), T(p.shift)
+
+        def launch(i):
+            i8.batched_gemm_i8(A, B, C, b, mu, sh, p.per_channel, p.relu)
+    return p.name, launch, ops, byts, sets
+
+
+def run(dev=None, cfgs=None, iters=50, graph=True, peak_tops=None, peak_gbs=None):
+    import torch
+    from . import binding as i8
+    dev = dev or torch.device("cuda", 0)
+    out = []
+    for name in (cfgs or ALL):
+        pname, launch, ops, byts, sets = _make(name, dev)
+        for i in range(max(5, sets)):
+            launch(i)
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            launch(i)
+        e1.record(); torch.cuda.synchronize()
+        us_loop = e0.elapsed_time(e1) / iters * 1e3
+        us_graph = None
+        if graph:
+            g = torch.cuda.CUDAGraph(); s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                launch(0); torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=s):
+                    for i in range(iters):
+                        launch(i)
+            torch.cuda.synchronize()
+            g.replay(); torch.cuda.synchronize()
+            e0.record(); g.replay(); e1.record(); torch.cuda.synchronize()
+            us_graph = e0.elapsed_time(e1) / iters * 1e3
+        us = min(us_loop, us_graph) if us_graph is not None else us_loop
+        rec = {"problem": pname, "us_per_launch": us, "us_loop": us_loop, "us_graph": us_graph, "tops": ops / us / 1e6,
+               "gbs": byts / us / 1e3, "path": i8.last_path(), "buffer_sets": sets,
+               "device_status": i8.last_device_status()}
+        if peak_tops and peak_gbs:
+            t_roof = max(ops / (peak_tops * 1e12), byts / (peak_gbs * 1e9)) * 1e6
+            rec["roofline_us"] = t_roof
+            rec["roofline_frac"] = t_roof / us
+            rec["bound"] = "tensor" if ops / (peak_tops * 1e12) >= byts / (peak_gbs * 1e9) else "hbm"
+        out.append(rec)
+    return out
+
+
+if __name__ == "__main__":
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--cfg", default=",".join(ALL))
+    ap.add_argument("--iters", type=int, default=50)
+    ap.add_argument("--no-graph", action="store_true")
+    a = ap.parse_args()
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    pk = os.path.join(root, "MEASURED_PEAKS.json")
+    peak_tops, peak_gbs = 2 * 1590.0, 6650.0
+    if os.path.exists(pk):
+        d = json.load(open(pk)); peak_tops, peak_gbs = 2 * d["bf16_tflops"], d["hbm_gbs"]
+    for r in run(cfgs=a.cfg.split(","), iters=a.iters, graph=not a.no_graph, peak_tops=peak_tops, peak_gbs=peak_gbs):
+        print(json.dumps(r), flush=True)

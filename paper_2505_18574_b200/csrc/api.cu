@@ -164,7 +164,7 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
     p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
     p.sched.group_m = 16;
     p.kl = kl;
-    p.wait_limit_ns = g_wait_limit_ns;
+    p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);   // SM clock stays below 2 GHz: at least the asked time
     p.dev_status = ctx->dev_status;
     if (conv) {
         switch (bn) {

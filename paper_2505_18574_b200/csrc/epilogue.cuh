@@ -72,13 +72,43 @@ __device__ __forceinline__ int32_t requant_fast(int32_t acc, int32_t bias, int32
     return (int32_t)__funnelshift_r(plo, phi, (uint32_t)shift);   // low word of p >> shift, shift in 0..31
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Shift-32 form.  When shift >= 1 and -2^(shift-1) <= mult < 2^(shift-1) (every scale below one half), the
+// multiplier can be pre-shifted: m2 = mult * 2^(32-shift) still fits in 32 bits and
+//     floor((t*mult + 2^(shift-1)) / 2^shift) = floor((t*m2 + 2^31) / 2^32),
+// the same rational number before the floor.  The result is then simply the HIGH word of one 64-bit
+// multiply-add, it always fits in 32 bits (|t*m2| <= 2^62), and the saturating pack finishes the clamp;
+// no window is needed.  The bias folds into the addend: with nb = -bias,
+//     max(acc + bias, 0)*m2 + 2^31 = max(acc, nb)*m2 + (bias*m2 + 2^31),
+// evaluated modulo 2^64 (the true value fits, so wrap-around in the partial sums is harmless).
+// Packed per output channel as int4 {m2, nb, addend low, addend high}.
+__device__ __forceinline__ bool make_shift32_const(int32_t bias, int32_t mult, int32_t shift, int relu, int4& out) {
+    out = make_int4(0, INT32_MIN, 0, 0);
+    if (shift < 1) return false;
+    const int32_t half = 1 << (shift - 1);
+    if (mult < -half || mult >= half) return false;
+    if (relu && bias == INT32_MIN) return false;        // -bias is not representable
+    const int32_t m2 = (int32_t)((uint32_t)mult << (32 - shift));
+    const unsigned long long c = (unsigned long long)((long long)bias * (long long)m2) + (1ull << 31);
+    out = make_int4(m2, relu ? -bias : INT32_MIN, (int32_t)(uint32_t)c, (int32_t)(uint32_t)(c >> 32));
+    return true;
+}
+
+template <bool RELU>
+__device__ __forceinline__ int32_t requant_shift32(int32_t acc, const int4& k) {
+    const int32_t t = RELU ? max(acc, k.y) : acc;
+    const unsigned long long c = (unsigned long long)(uint32_t)k.z | ((unsigned long long)(uint32_t)k.w << 32);
+    const unsigned long long p = (unsigned long long)((long long)t * (long long)k.x) + c;
+    return (int32_t)(uint32_t)(p >> 32);
+}
+
 // Saturate four 32-bit values to int8 and pack them, v0 in the lowest byte.
+// cvt.pack.sat.s8.s32.b32 d, a, b, c  gives  d = (c << 16) | (sat8(a) << 8) | sat8(b).
 __device__ __forceinline__ uint32_t pack_sat4(int32_t v0, int32_t v1, int32_t v2, int32_t v3) {
-    v0 = min(max(v0, -128), 127);
-    v1 = min(max(v1, -128), 127);
-    v2 = min(max(v2, -128), 127);
-    v3 = min(max(v3, -128), 127);
-    return ((uint32_t)v0 & 0xffu) | (((uint32_t)v1 & 0xffu) << 8) | (((uint32_t)v2 & 0xffu) << 16) | ((uint32_t)v3 << 24);
+    uint32_t hi, d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(v3), "r"(v2), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(v1), "r"(v0), "r"(hi));
+    return d;
 }
 
 }  // namespace i8

@@ -58,7 +58,7 @@ struct GemmTcParams {
     int c_vec_ok;               // C and ldc are 16-byte aligned: full chunks go out as 16-byte stores
     TileSched sched;
     KLoop kl;
-    uint64_t wait_limit_ns;
+    long long wait_limit_cycles;
     unsigned* dev_status;
 };
 
@@ -68,8 +68,8 @@ struct TcSmem {
     static constexpr int B_BYTES = BN * BK;
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-    static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // 6 int32 arrays of BN entries
-    static constexpr int OFF_BAR = OFF_CONST + 6 * BN * 4;           // full[S], empty[S], acc_full[2], acc_empty[2]
+    static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // int4[BN] shift-32 constants, then 6 int32[BN] arrays
+    static constexpr int OFF_BAR = OFF_CONST + 10 * BN * 4;          // full[S], empty[S], acc_full[2], acc_empty[2]
     static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 4) * 8;  // tensor-memory base, stop flag
     static constexpr int TOTAL = OFF_MISC + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;                   // slack to align the base to 1024 bytes
@@ -92,6 +92,19 @@ __device__ __forceinline__ void epilogue_chunk(const int32_t (&v)[32], const int
         const int32_t r1 = requant_fast(v[4 * j + 1], bi.y, lo.y, hi.y, mu.y, sh.y, rn.y);
         const int32_t r2 = requant_fast(v[4 * j + 2], bi.z, lo.z, hi.z, mu.z, sh.z, rn.z);
         const int32_t r3 = requant_fast(v[4 * j + 3], bi.w, lo.w, hi.w, mu.w, sh.w, rn.w);
+        out[j] = pack_sat4(r0, r1, r2, r3);
+    }
+}
+
+// Same chunk in the shift-32 form: one 16-byte constant load, at most one max, one widening multiply-add per output.
+template <bool RELU>
+__device__ __forceinline__ void epilogue_chunk_shift32(const int32_t (&v)[32], const int4* s_k, int c0, uint32_t (&out)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+        const int32_t r0 = requant_shift32<RELU>(v[4 * j + 0], s_k[c0 + 4 * j + 0]);
+        const int32_t r1 = requant_shift32<RELU>(v[4 * j + 1], s_k[c0 + 4 * j + 1]);
+        const int32_t r2 = requant_shift32<RELU>(v[4 * j + 2], s_k[c0 + 4 * j + 2]);
+        const int32_t r3 = requant_shift32<RELU>(v[4 * j + 3], s_k[c0 + 4 * j + 3]);
         out[j] = pack_sat4(r0, r1, r2, r3);
     }
 }
@@ -126,7 +139,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const uint32_t sbase = raw + pad;
 
     const uint32_t sA = sbase + L::OFF_A, sB = sbase + L::OFF_B;
-    int32_t* s_bias = reinterpret_cast<int32_t*>(smem + L::OFF_CONST);
+    int4* s_k32 = reinterpret_cast<int4*>(smem + L::OFF_CONST);
+    int32_t* s_bias = reinterpret_cast<int32_t*>(smem + L::OFF_CONST) + 4 * BN;
     int32_t* s_lo = s_bias + BN;
     int32_t* s_hi = s_lo + BN;
     int32_t* s_mult = s_hi + BN;
@@ -140,7 +154,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     volatile int* s_stop = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const WaitEnv env{s_stop, p.dev_status, p.wait_limit_ns};
+    const WaitEnv env{s_stop, p.dev_status, p.wait_limit_cycles};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) {
@@ -217,7 +231,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 // stopping early: let every copy this thread started land before the CTA retires
                 for (int s = 0; s < STAGES; s++)
                     if (issued & (1u << s))
-                        if (!mbar_wait_drain(bar_full + 8 * s, (issued_phase >> s) & 1u, p.wait_limit_ns))
+                        if (!mbar_wait_drain(bar_full + 8 * s, (issued_phase >> s) & 1u, p.wait_limit_cycles))
                             atomicCAS(p.dev_status, 0u, (unsigned)DEV_TIMEOUT_DRAIN);
             }
         }
@@ -273,6 +287,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int quarter = warp & 3;                   // a warp may only read lanes 32*(warp%4) .. +31
         const int cgroup = (warp - 2) >> 2;             // which share of the columns this warp handles
         int ab = 0, cached_n_blk = -1;
+        bool shift32 = false;                           // every channel of the cached block admits the shift-32 form
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < sched.num_tiles; tile += gridDim.x) {
             int m_blk, n_blk;
@@ -283,6 +298,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tc_fence_after();
             const int n0 = n_blk * BN;
             if (n_blk != cached_n_blk) {
+                bool all32 = true;
                 for (int c = etid; c < BN; c += EPI_THREADS) {
                     const int n = n0 + c;
                     int32_t bias = 0, mult = 0, shift = 0;
@@ -294,9 +310,12 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const ChanConst cc = make_chan_const(mult, shift, p.relu);
                     s_bias[c] = bias; s_lo[c] = cc.lo; s_hi[c] = cc.hi;
                     s_mult[c] = cc.mult; s_shift[c] = cc.shift; s_rnd[c] = cc.rnd;
+                    int4 k32;
+                    all32 = make_shift32_const(bias, mult, shift, p.relu, k32) && all32;
+                    s_k32[c] = k32;
                 }
                 cached_n_blk = n_blk;
-                named_barrier(2, EPI_THREADS);
+                shift32 = named_barrier_and(2, EPI_THREADS, all32);
             }
             const int row = m_blk * BM + quarter * 32 + lane;
             int8_t* crow = p.C + (int64_t)row * p.ldc;
@@ -310,7 +329,12 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 tmem_ld_32x32(t0 + c0, v);
                 tmem_ld_wait();
                 uint32_t out[8];
-                epilogue_chunk(v, s_bias, s_lo, s_hi, s_mult, s_shift, s_rnd, c0, out);
+                if (shift32) {
+                    if (p.relu) epilogue_chunk_shift32<true>(v, s_k32, c0, out);
+                    else epilogue_chunk_shift32<false>(v, s_k32, c0, out);
+                } else {
+                    epilogue_chunk(v, s_bias, s_lo, s_hi, s_mult, s_shift, s_rnd, c0, out);
+                }
                 if (row < p.M) store_row_chunk(crow, n, p.N, p.c_vec_ok != 0, out);
             }
             tc_fence_before();

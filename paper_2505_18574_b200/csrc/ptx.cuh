@@ -63,19 +63,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 struct WaitEnv {
     volatile int* stop;        // shared-memory flag: somebody gave up, everybody leaves
     unsigned* dev_status;      // global status word
-    uint64_t limit_ns;         // longest single wait
+    long long limit_cycles;    // longest single wait, in SM clock cycles
 };
 
 // Wait for `bar` to complete the phase with the given parity.  Returns false (and raises the CTA's stop
 // flag plus the global status word) when the limit expires, or when another thread already gave up.
+// The clock is only consulted after a burst of failed polls, so an ordinary short wait costs nothing extra.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitEnv& env, unsigned code) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+#pragma unroll 1
+    for (int i = 0; i < 64; i++)
+        if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0xff) == 0) {
+        if ((++spins & 0x3f) == 0) {
             if (*env.stop) return false;
-            if (globaltimer_ns() - t0 > env.limit_ns) {
+            if (clock64() - t0 > env.limit_cycles) {
                 *env.stop = 1;
                 atomicCAS(env.dev_status, 0u, code);
                 return false;
@@ -86,12 +89,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
 }
 
 // Same wait, but it ignores the stop flag: used while stopping, to let copies already in flight land.
-__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
+__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity, long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+    const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0xff) == 0 && globaltimer_ns() - t0 > limit_ns) return false;
+        if ((++spins & 0x3f) == 0 && clock64() - t0 > limit_cycles) return false;
     }
     return true;
 }
