@@ -186,99 +186,103 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const uint32_t a_sub_bytes = BM * kl.cb, b_sub_bytes = BN * kl.cb;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0, issued = 0, issued_phase = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
-                int m_blk, n_blk;
-                sched.map(tile, m_blk, n_blk);
-                int w0 = 0, h0 = 0, img = 0;
-                if (CONV) {
-                    // first output pixel of the tile -> position of filter tap (0,0) in the input image
-                    const int m0 = m_blk * BM;
-                    const int pq = kl.P * kl.Q;
-                    img = m0 / pq;
-                    const int rem = m0 - img * pq;
-                    const int op = rem / kl.Q, oq = rem - op * kl.Q;
-                    h0 = op * kl.stride_h - kl.pad_h;
-                    w0 = oq * kl.stride_w - kl.pad_w;
-                }
-                int c_idx = 0, fs = 0, fr = 0;      // convolution: channel block, filter column, filter row
-                for (int kbi = 0; kbi < kl.num_kblocks;) {
-                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
-                    const int nb = min(kl.nsub, kl.num_kblocks - kbi);
-                    const uint32_t full = bar_full + 8 * stage;
-                    mbar_expect_tx(full, nb * (a_sub_bytes + b_sub_bytes));
-                    for (int j = 0; j < nb; j++, kbi++) {
-                        const uint32_t dstA = sA + stage * L::A_BYTES + j * a_sub_bytes;
-                        const uint32_t dstB = sB + stage * L::B_BYTES + j * b_sub_bytes;
-                        if (CONV) {
-                            tma_load_im2col_4d(dstA, &tmA, full, c_idx * kl.cb, w0, h0, img, (uint16_t)fs, (uint16_t)fr);
-                            if (++c_idx == kl.cblocks) { c_idx = 0; if (++fs == kl.S) { fs = 0; ++fr; } }
-                        } else {
-                            tma_load_2d(dstA, &tmA, full, kbi * BK, m_blk * BM);
-                        }
-                        tma_load_2d(dstB, &tmB, full, kbi * kl.cb, n_blk * BN);
+        // ------------------------------------------------------------------ producer (whole warp loops, one lane issues)
+        int stage = 0;
+        uint32_t phase = 0, issued = 0, issued_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
+            int m_blk, n_blk;
+            sched.map(tile, m_blk, n_blk);
+            int w0 = 0, h0 = 0, img = 0;
+            if (CONV) {
+                // first output pixel of the tile -> position of filter tap (0,0) in the input image
+                const int m0 = m_blk * BM;
+                const int pq = kl.P * kl.Q;
+                img = m0 / pq;
+                const int rem = m0 - img * pq;
+                const int op = rem / kl.Q, oq = rem - op * kl.Q;
+                h0 = op * kl.stride_h - kl.pad_h;
+                w0 = oq * kl.stride_w - kl.pad_w;
+            }
+            int c_idx = 0, fs = 0, fr = 0;      // convolution: channel block, filter column, filter row
+            for (int kbi = 0; kbi < kl.num_kblocks;) {
+                if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                const int nb = min(kl.nsub, kl.num_kblocks - kbi);
+                const uint32_t full = bar_full + 8 * stage;
+                const bool leader = elect_one();
+                if (leader) mbar_expect_tx(full, nb * (a_sub_bytes + b_sub_bytes));
+                for (int j = 0; j < nb; j++, kbi++) {
+                    const uint32_t dstA = sA + stage * L::A_BYTES + j * a_sub_bytes;
+                    const uint32_t dstB = sB + stage * L::B_BYTES + j * b_sub_bytes;
+                    if (CONV) {
+                        if (leader) tma_load_im2col_4d(dstA, &tmA, full, c_idx * kl.cb, w0, h0, img, (uint16_t)fs, (uint16_t)fr);
+                        if (++c_idx == kl.cblocks) { c_idx = 0; if (++fs == kl.S) { fs = 0; ++fr; } }
+                    } else {
+                        if (leader) tma_load_2d(dstA, &tmA, full, kbi * BK, m_blk * BM);
                     }
-                    issued |= 1u << stage;
-                    issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    if (leader) tma_load_2d(dstB, &tmB, full, kbi * kl.cb, n_blk * BN);
                 }
+                issued |= 1u << stage;
+                issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
+                if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
-            if (*s_stop) {
-                // stopping early: let every copy this thread started land before the CTA retires
-                for (int s = 0; s < STAGES; s++)
-                    if (issued & (1u << s))
-                        if (!mbar_wait_drain(bar_full + 8 * s, (issued_phase >> s) & 1u, p.wait_limit_cycles))
-                            atomicCAS(p.dev_status, 0u, (unsigned)DEV_TIMEOUT_DRAIN);
-            }
+        }
+        if (*s_stop) {
+            // stopping early: let every copy this warp started land before the CTA retires
+            for (int s = 0; s < STAGES; s++)
+                if (issued & (1u << s))
+                    if (!mbar_wait_drain(bar_full + 8 * s, (issued_phase >> s) & 1u, p.wait_limit_cycles))
+                        atomicCAS(p.dev_status, 0u, (unsigned)DEV_TIMEOUT_DRAIN);
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_i8(BM, BN, 0, 0);
-            // K-major operands: rows cb bytes apart, swizzled over cb bytes, 8-row groups 8*cb bytes apart;
-            // a 32-byte step along K inside a swizzle row is a plain address offset.
-            const uint64_t swz = kl.cb == 128 ? SWZ_128B : (kl.cb == 64 ? SWZ_64B : SWZ_32B);
-            const uint32_t sbo = 8 * kl.cb;
-            int stage = 0, ab = 0;
-            uint32_t phase = 0, acc_phase = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
-                if (!mbar_wait(bar_acc_empty + 8 * ab, acc_phase ^ 1, env, DEV_TIMEOUT_MMA_ACC)) break;
+        // ------------------------------------------------------------------ MMA issuer (whole warp loops, one lane issues)
+        constexpr uint32_t idesc = make_idesc_i8(BM, BN, 0, 0);
+        // K-major operands: rows cb bytes apart, swizzled over cb bytes, 8-row groups 8*cb bytes apart;
+        // a 32-byte step along K inside a swizzle row is a plain address offset.
+        const uint64_t swz = kl.cb == 128 ? SWZ_128B : (kl.cb == 64 ? SWZ_64B : SWZ_32B);
+        const uint32_t sbo = 8 * kl.cb;
+        const uint64_t desc_hi = make_smem_desc(0, 16, sbo, swz);   // everything but the start address
+        int stage = 0, ab = 0;
+        uint32_t phase = 0, acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
+            if (!mbar_wait_warp(bar_acc_empty + 8 * ab, acc_phase ^ 1, env, DEV_TIMEOUT_MMA_ACC)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + ab * BN;
+            uint32_t accumulate = 0;
+            for (int kbi = 0; kbi < kl.num_kblocks;) {
+                if (!mbar_wait_warp(bar_full + 8 * stage, phase, env, DEV_TIMEOUT_MMA_FULL)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + ab * BN;
-                uint32_t accumulate = 0;
-                for (int kbi = 0; kbi < kl.num_kblocks;) {
-                    if (!mbar_wait(bar_full + 8 * stage, phase, env, DEV_TIMEOUT_MMA_FULL)) { ok = false; break; }
-                    tc_fence_after();
-                    const int nb = min(kl.nsub, kl.num_kblocks - kbi);
-                    for (int j = 0; j < nb; j++, kbi++) {
-                        const uint32_t a0 = sA + stage * L::A_BYTES + j * a_sub_bytes;
-                        const uint32_t b0 = sB + stage * L::B_BYTES + j * b_sub_bytes;
-                        int ksteps = kl.cb / UMMA_K;
-                        if (!CONV) {                       // GEMM: the last block may be ragged in K
-                            const int rem = p.K - kbi * BK;
-                            if (rem < BK) ksteps = (rem + UMMA_K - 1) / UMMA_K;
-                        }
+                const int nb = min(kl.nsub, kl.num_kblocks - kbi);
+                const bool leader = elect_one();
+                for (int j = 0; j < nb; j++, kbi++) {
+                    const uint32_t a0 = sA + stage * L::A_BYTES + j * a_sub_bytes;
+                    const uint32_t b0 = sB + stage * L::B_BYTES + j * b_sub_bytes;
+                    int ksteps = kl.cb / UMMA_K;
+                    if (!CONV) {                       // GEMM: the last block may be ragged in K
+                        const int rem = p.K - kbi * BK;
+                        if (rem < BK) ksteps = (rem + UMMA_K - 1) / UMMA_K;
+                    }
+                    if (leader) {
                         for (int k = 0; k < ksteps; k++) {
-                            const uint64_t ad = make_smem_desc(a0 + k * UMMA_K, 16, sbo, swz);
-                            const uint64_t bd = make_smem_desc(b0 + k * UMMA_K, 16, sbo, swz);
+                            const uint64_t ad = desc_hi | (uint64_t)(((a0 + k * UMMA_K) & 0x3FFFFu) >> 4);
+                            const uint64_t bd = desc_hi | (uint64_t)(((b0 + k * UMMA_K) & 0x3FFFFu) >> 4);
                             mma_i8_ss(d_tmem, ad, bd, idesc, accumulate);
                             accumulate = 1;
                         }
                     }
-                    tc_commit(bar_empty + 8 * stage);   // slot reusable once these MMAs have read it
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    accumulate = 1;
                 }
-                if (!ok) break;
-                tc_commit(bar_acc_full + 8 * ab);       // accumulator complete
-                ab ^= 1;
-                if (ab == 0) acc_phase ^= 1;
+                if (leader) tc_commit(bar_empty + 8 * stage);   // slot reusable once these MMAs have read it
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
+            if (!ok) break;
+            if (elect_one()) tc_commit(bar_acc_full + 8 * ab);  // accumulator complete
+            __syncwarp();
+            ab ^= 1;
+            if (ab == 0) acc_phase ^= 1;
         }
         __syncwarp();
     } else {

@@ -99,6 +99,25 @@ __device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity, l
     return true;
 }
 
+// Warp-uniform variant: every lane of a converged warp polls, and all lanes leave with the same answer.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitEnv& env, unsigned code) {
+    const bool ok = mbar_wait(bar, parity, env, code);
+    return __all_sync(0xffffffffu, ok);
+}
+
+// True in exactly one lane of a converged warp.  Keeping the whole warp in a role's loop and electing a
+// lane only around the issuing instructions lets the compiler hold descriptors and coordinates in uniform
+// registers, which the TMA and tcgen05 instructions take directly.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 // Barrier among `nthreads` threads (a multiple of 32) that also ANDs a predicate over them.
 __device__ __forceinline__ bool named_barrier_and(int id, int nthreads, bool pred) {
     uint32_t out;
