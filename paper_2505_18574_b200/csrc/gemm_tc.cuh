@@ -153,7 +153,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC);
     volatile int* s_stop = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // broadcast from lane 0 so the compiler can treat the role index as warp-uniform
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
+    const int lane = threadIdx.x & 31;
     const WaitEnv env{s_stop, p.dev_status, p.wait_limit_cycles};
 
     if (threadIdx.x == 0) {
@@ -179,7 +181,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *s_tmem;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *s_tmem, 0);   // same value in every lane, known uniform
 
     const TileSched sched = p.sched;
     const KLoop kl = p.kl;
