@@ -9,6 +9,7 @@
 #include <mutex>
 
 #include "../../include/i8ops.h"
+#include "batched_tc.cuh"
 #include "gemm_tc.cuh"
 #include "generic.cuh"
 
@@ -222,6 +223,45 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     return run_tc(ctx, true, tmA, kl, bn, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
 }
 
+// Paired small-tile path: problems with M, N, K <= 64, two per MMA.
+static int run_batched_pair(DeviceCtx* ctx, const int8_t* A, int64_t a_rs, int64_t a_bs, const int8_t* B, int64_t b_ld,
+                            int64_t b_bs, int b_mn_major, int8_t* C, int64_t ldc, int64_t c_bs, const int32_t* bias,
+                            int64_t bias_bs, const int32_t* mult, const int32_t* shift, int per_channel, int batch, int M,
+                            int N, int K, int relu, cudaStream_t st) {
+    CUtensorMap tmA, tmB;
+    const uint32_t box[3] = {64, 64, 2};
+    {
+        const uint64_t dims[3] = {(uint64_t)K, (uint64_t)M, (uint64_t)batch};
+        const uint64_t str[2] = {(uint64_t)a_rs, (uint64_t)a_bs};
+        int rc = make_tmap(&tmA, A, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_64B);
+        if (rc) return rc;
+    }
+    {
+        const uint64_t dimsK[3] = {(uint64_t)K, (uint64_t)N, (uint64_t)batch};   // K contiguous: rows are output columns
+        const uint64_t dimsN[3] = {(uint64_t)N, (uint64_t)K, (uint64_t)batch};   // N contiguous: rows are K
+        const uint64_t str[2] = {(uint64_t)b_ld, (uint64_t)b_bs};
+        int rc = make_tmap(&tmB, B, 3, b_mn_major ? dimsN : dimsK, str, box, CU_TENSOR_MAP_SWIZZLE_64B);
+        if (rc) return rc;
+    }
+    BatchedPairParams p;
+    p.C = C; p.ldc = ldc; p.c_bs = c_bs; p.bias = bias; p.bias_bs = bias_bs; p.mult = mult; p.shift = shift;
+    p.per_channel = per_channel; p.relu = relu; p.batch = batch; p.M = M; p.N = N; p.K = K;
+    p.b_mn_major = b_mn_major;
+    p.c_vec_ok = aligned16(C) && ldc % 16 == 0 && c_bs % 16 == 0;
+    p.bias_vec_ok = bias && aligned16(bias) && bias_bs % 4 == 0;
+    p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);
+    p.dev_status = ctx->dev_status;
+    if (!ctx->attr_set[6]) {
+        CUDA_TRY(cudaFuncSetAttribute(batched_pair_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::DYN_BYTES));
+        ctx->attr_set[6] = true;
+    }
+    const int pairs = (batch + 1) / 2;
+    const int grid = pairs < ctx->sm_count ? pairs : ctx->sm_count;
+    batched_pair_i8_kernel<<<grid, PAIR_THREADS, PairSmem::DYN_BYTES, st>>>(tmA, tmB, p);
+    CUDA_TRY(cudaGetLastError());
+    return I8_OK;
+}
+
 static int run_gemm_generic(const GenericGemmParams& p, cudaStream_t st) {
     const int64_t total = (int64_t)p.batch * p.M * p.N;
     int64_t blocks = (total + 255) / 256;
@@ -295,6 +335,17 @@ int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs, c
     rc = get_ctx(&ctx);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    if (g_path_mode != 1 && M <= 64 && N <= 64 && K >= 1 && K <= 64 && a_cs == 1 && aligned16(A) && aligned16(B) &&
+        a_rs % 16 == 0 && a_bs % 16 == 0 && b_bs % 16 == 0 && a_rs >= K) {
+        const bool b_n_contig = b_cs == 1 && b_rs % 16 == 0 && b_rs >= N;      // row-major B: MN-major operand
+        const bool b_k_contig = b_rs == 1 && b_cs % 16 == 0 && b_cs >= K;      // column-major B: K-major operand
+        if (b_k_contig || b_n_contig) {
+            rc = run_batched_pair(ctx, A, a_rs, a_bs, B, b_k_contig ? b_cs : b_rs, b_bs, b_k_contig ? 0 : 1, C, ldc, c_bs,
+                                  bias, bias_bs, mult, shift, per_channel, batch, M, N, K, relu, st);
+            if (rc == I8_OK) t_last_path = I8_PATH_SMALL;
+            return rc;
+        }
+    }
     GenericGemmParams g{A, a_rs, a_cs, a_bs, B, b_rs, b_cs, b_bs, C, ldc, c_bs, bias, bias_bs, mult, shift, per_channel, relu,
                         batch, M, N, K};
     rc = run_gemm_generic(g, st);

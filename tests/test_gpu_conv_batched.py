@@ -116,8 +116,52 @@ def test_batched_shapes(batch, M, N, K, ppb):
         H.assert_same(H.batched_gpu(p), want, f"{p.name} mode {mode}")
 
 
+@pytest.mark.parametrize("batch,M,N,K", [(2, 64, 64, 64), (7, 64, 64, 64), (1, 64, 64, 64), (6, 64, 32, 64), (5, 17, 64, 48),
+                                         (4, 64, 16, 16), (9, 40, 48, 32), (300, 64, 64, 64), (3, 1, 64, 64)])
+@pytest.mark.parametrize("b_col_major", [False, True])
+def test_batched_small_tile_path(batch, M, N, K, b_col_major):
+    """Paired small-tile kernel: row-major B goes through an MN-major descriptor, column-major B through a K-major one."""
+    import torch
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_batched(batch, M, N, K, 600 + batch + M + N + K)
+    p.shift[:] = 13
+    want = H.batched_oracle(p)
+    A = torch.from_numpy(p.A).cuda()
+    if b_col_major:
+        B = torch.from_numpy(np.ascontiguousarray(p.B.transpose(0, 2, 1))).cuda().transpose(1, 2)   # (batch, K, N) view, K contiguous
+    else:
+        B = torch.from_numpy(p.B).cuda()
+    C = torch.full((batch, M, N), 0x5A, dtype=torch.int8, device="cuda")
+    i8.set_path(0)
+    i8.batched_gemm_i8(A, B, C, torch.from_numpy(p.bias).cuda(), torch.from_numpy(p.mult).cuda(), torch.from_numpy(p.shift).cuda(),
+                       p.per_channel, p.relu)
+    assert i8.last_device_status() == 0
+    assert i8.last_path() == i8.PATH_SMALL
+    H.assert_same(C.cpu().numpy(), want, f"{p.name} b_col_major={b_col_major}")
+
+
+@pytest.mark.parametrize("mult,shift,relu,per_channel", [(1, 0, 0, 0), (-3, 1, 1, 0), (2147483647, 31, 0, 0), (20000, 20, 1, 1), (0, 7, 0, 0)])
+def test_batched_small_tile_scales(mult, shift, relu, per_channel):
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_batched(5, 64, 64, 64, 9, relu=relu)
+    if per_channel:
+        rng = np.random.default_rng(4)
+        p.mult = rng.integers(-(1 << 15), 1 << 15, size=64, dtype=np.int32)
+        p.shift = rng.integers(0, 25, size=64, dtype=np.int32)
+        p.per_channel = 1
+    else:
+        p.mult[:] = mult; p.shift[:] = shift
+    want = H.batched_oracle(p)
+    i8.set_path(0)
+    got = H.batched_gpu(p)
+    assert i8.last_path() == i8.PATH_SMALL
+    H.assert_same(got, want, p.name)
+
+
 def test_config4b_batched():
+    import paper_2505_18574_b200 as i8
     p = inputs.config4b()
     want = H.batched_oracle(p)
     H.assert_same(H.batched_gpu(p), want, p.name)
+    assert i8.last_path() == i8.PATH_SMALL
     H.not_degenerate(want)
