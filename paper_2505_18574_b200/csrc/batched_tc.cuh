@@ -54,6 +54,54 @@ struct PairSmem {
     static constexpr int TMEM_COLS = 128 * PAIR_ACC;                          // 512
 };
 
+// 32 consecutive bias entries starting at column n0 (zeros where there is no bias or no such column).
+__device__ __forceinline__ void load_bias32(const int32_t* brow, int n0, int N, bool vec_ok, int4 (&bq)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) bq[j] = make_int4(0, 0, 0, 0);
+    if (!brow) return;
+    if (vec_ok && n0 + 32 <= N) {
+#pragma unroll
+        for (int j = 0; j < 8; j++) bq[j] = __ldg(reinterpret_cast<const int4*>(brow + n0) + j);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            const int c = n0 + 4 * j;
+            if (c + 0 < N) bq[j].x = __ldg(brow + c + 0);
+            if (c + 1 < N) bq[j].y = __ldg(brow + c + 1);
+            if (c + 2 < N) bq[j].z = __ldg(brow + c + 2);
+            if (c + 3 < N) bq[j].w = __ldg(brow + c + 3);
+        }
+    }
+}
+
+// Epilogue arithmetic of one 32-column chunk.  MODE 0: shift-32 form, one multiplier for all channels;
+// MODE 1: shift-32 form, per-channel multipliers from shared memory; MODE 2: window form (any scale).
+template <int MODE, bool RELU>
+__device__ __forceinline__ void pair_chunk(const int32_t (&v)[32], const int4 (&bq)[8], int n0, int32_t m2_shared,
+                                           const int32_t* s_m2, const int32_t* s_lo, const int32_t* s_hi, const int32_t* s_mult,
+                                           const int32_t* s_shift, const int32_t* s_rnd, uint32_t (&out)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+        const int bb[4] = {bq[j].x, bq[j].y, bq[j].z, bq[j].w};
+        int32_t r[4];
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+            const int c = n0 + 4 * j + e;
+            if (MODE == 2) {
+                r[e] = requant_fast(v[4 * j + e], bb[e], s_lo[c], s_hi[c], s_mult[c], s_shift[c], s_rnd[c]);
+            } else {
+                // high word of max(acc + bias, 0) * m2 + 2^31
+                int32_t tt = v[4 * j + e] + bb[e];
+                if (RELU) tt = max(tt, 0);
+                const int32_t m2 = MODE == 1 ? s_m2[c] : m2_shared;
+                const unsigned long long pr = (unsigned long long)((long long)tt * (long long)m2) + (1ull << 31);
+                r[e] = (int32_t)(uint32_t)(pr >> 32);
+            }
+        }
+        out[j] = pack_sat4(r[0], r[1], r[2], r[3]);
+    }
+}
+
 __global__ void __launch_bounds__(PAIR_THREADS, 1)
 batched_pair_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const BatchedPairParams p) {
     using L = PairSmem;
@@ -187,14 +235,17 @@ batched_pair_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         int seq = 0;                                       // index of this CTA's pair, to pick every PAIR_ACC-th one
         for (int t = blockIdx.x; t < num_pairs; t += gridDim.x, seq++) {
             if ((seq % PAIR_ACC) != g) continue;
+            const int prob = 2 * t + which;
+            const bool live = prob < p.batch && row < p.M;
+            int8_t* crow = p.C + (int64_t)prob * p.c_bs + (int64_t)row * p.ldc;
+            const int32_t* brow = (p.bias && prob < p.batch) ? p.bias + (int64_t)prob * p.bias_bs : nullptr;
+            // the bias of the first 32 columns does not depend on the product: fetch it before waiting
+            int4 bq[8];
+            load_bias32(brow, 0, p.N, p.bias_vec_ok != 0, bq);
             bool ok = mbar_wait(bar_acc_full + 8 * g, acc_phase, env, DEV_TIMEOUT_EPILOGUE);
             ok = named_barrier_and(1 + g, 128, ok);
             if (!ok) break;
             tc_fence_after();
-            const int prob = 2 * t + which;
-            const bool live = prob < p.batch && row < p.M;
-            int8_t* crow = p.C + (int64_t)prob * p.c_bs + (int64_t)row * p.ldc;
-            const int32_t* brow = p.bias ? p.bias + (int64_t)prob * p.bias_bs : nullptr;
             const uint32_t t0 = tmem_base + g * 128 + which * 64 + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
             for (int ch = 0; ch < 2; ch++) {
@@ -204,37 +255,18 @@ batched_pair_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                 tmem_ld_32x32(t0 + n0, v);
                 tmem_ld_wait();
                 uint32_t out[8];
-#pragma unroll
-                for (int j = 0; j < 8; j++) {
-                    int4 b4 = make_int4(0, 0, 0, 0);
-                    if (brow && prob < p.batch) {
-                        if (p.bias_vec_ok && n0 + 4 * j + 4 <= p.N) {
-                            b4 = __ldg(reinterpret_cast<const int4*>(brow + n0 + 4 * j));
-                        } else {
-                            if (n0 + 4 * j + 0 < p.N) b4.x = __ldg(brow + n0 + 4 * j + 0);
-                            if (n0 + 4 * j + 1 < p.N) b4.y = __ldg(brow + n0 + 4 * j + 1);
-                            if (n0 + 4 * j + 2 < p.N) b4.z = __ldg(brow + n0 + 4 * j + 2);
-                            if (n0 + 4 * j + 3 < p.N) b4.w = __ldg(brow + n0 + 4 * j + 3);
-                        }
+                if (all32) {
+                    if (p.per_channel) {
+                        if (p.relu) pair_chunk<1, true>(v, bq, n0, m2_shared, s_m2, s_lo, s_hi, s_mult, s_shift, s_rnd, out);
+                        else pair_chunk<1, false>(v, bq, n0, m2_shared, s_m2, s_lo, s_hi, s_mult, s_shift, s_rnd, out);
+                    } else {
+                        if (p.relu) pair_chunk<0, true>(v, bq, n0, m2_shared, s_m2, s_lo, s_hi, s_mult, s_shift, s_rnd, out);
+                        else pair_chunk<0, false>(v, bq, n0, m2_shared, s_m2, s_lo, s_hi, s_mult, s_shift, s_rnd, out);
                     }
-                    const int bb[4] = {b4.x, b4.y, b4.z, b4.w};
-                    int32_t r[4];
-#pragma unroll
-                    for (int e = 0; e < 4; e++) {
-                        const int c = n0 + 4 * j + e;
-                        if (all32) {
-                            // high word of max(acc + bias, 0) * m2 + 2^31
-                            int32_t tt = v[4 * j + e] + bb[e];
-                            if (p.relu) tt = max(tt, 0);
-                            const int32_t m2 = p.per_channel ? s_m2[c] : m2_shared;
-                            const unsigned long long pr = (unsigned long long)((long long)tt * (long long)m2) + (1ull << 31);
-                            r[e] = (int32_t)(uint32_t)(pr >> 32);
-                        } else {
-                            r[e] = requant_fast(v[4 * j + e], bb[e], s_lo[c], s_hi[c], s_mult[c], s_shift[c], s_rnd[c]);
-                        }
-                    }
-                    out[j] = pack_sat4(r[0], r[1], r[2], r[3]);
+                } else {
+                    pair_chunk<2, false>(v, bq, n0, m2_shared, s_m2, s_lo, s_hi, s_mult, s_shift, s_rnd, out);
                 }
+                if (ch == 0 && p.N > 32) load_bias32(brow, 32, p.N, p.bias_vec_ok != 0, bq);   // next chunk's bias, in flight during the stores
                 if (live) {
                     if (p.c_vec_ok && n0 + 32 <= p.N) {
                         uint4* dst = reinterpret_cast<uint4*>(crow + n0);
