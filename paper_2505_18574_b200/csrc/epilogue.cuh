@@ -78,27 +78,22 @@ __device__ __forceinline__ int32_t requant_fast(int32_t acc, int32_t bias, int32
 //     floor((t*mult + 2^(shift-1)) / 2^shift) = floor((t*m2 + 2^31) / 2^32),
 // the same rational number before the floor.  The result is then simply the HIGH word of one 64-bit
 // multiply-add, it always fits in 32 bits (|t*m2| <= 2^62), and the saturating pack finishes the clamp;
-// no window is needed.  The bias folds into the addend: with nb = -bias,
-//     max(acc + bias, 0)*m2 + 2^31 = max(acc, nb)*m2 + (bias*m2 + 2^31),
-// evaluated modulo 2^64 (the true value fits, so wrap-around in the partial sums is harmless).
-// Packed per output channel as int4 {m2, nb, addend low, addend high}.
-__device__ __forceinline__ bool make_shift32_const(int32_t bias, int32_t mult, int32_t shift, int relu, int4& out) {
-    out = make_int4(0, INT32_MIN, 0, 0);
+// no window is needed.  Per output: one add (bias), at most one max (ReLU), one widening multiply-add.
+// Per output channel only two words are needed, the bias and m2 (one word when the multiplier is shared).
+__device__ __forceinline__ bool make_shift32_mult(int32_t mult, int32_t shift, int32_t& m2) {
+    m2 = 0;
     if (shift < 1) return false;
     const int32_t half = 1 << (shift - 1);
     if (mult < -half || mult >= half) return false;
-    if (relu && bias == INT32_MIN) return false;        // -bias is not representable
-    const int32_t m2 = (int32_t)((uint32_t)mult << (32 - shift));
-    const unsigned long long c = (unsigned long long)((long long)bias * (long long)m2) + (1ull << 31);
-    out = make_int4(m2, relu ? -bias : INT32_MIN, (int32_t)(uint32_t)c, (int32_t)(uint32_t)(c >> 32));
+    m2 = (int32_t)((uint32_t)mult << (32 - shift));
     return true;
 }
 
 template <bool RELU>
-__device__ __forceinline__ int32_t requant_shift32(int32_t acc, const int4& k) {
-    const int32_t t = RELU ? max(acc, k.y) : acc;
-    const unsigned long long c = (unsigned long long)(uint32_t)k.z | ((unsigned long long)(uint32_t)k.w << 32);
-    const unsigned long long p = (unsigned long long)((long long)t * (long long)k.x) + c;
+__device__ __forceinline__ int32_t requant_shift32(int32_t acc, int32_t bias, int32_t m2) {
+    int32_t t = acc + bias;
+    if (RELU) t = max(t, 0);
+    const unsigned long long p = (unsigned long long)((long long)t * (long long)m2) + (1ull << 31);
     return (int32_t)(uint32_t)(p >> 32);
 }
 

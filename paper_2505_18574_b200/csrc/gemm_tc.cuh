@@ -68,8 +68,8 @@ struct TcSmem {
     static constexpr int B_BYTES = BN * BK;
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-    static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // int4[BN] shift-32 constants, then 6 int32[BN] arrays
-    static constexpr int OFF_BAR = OFF_CONST + 10 * BN * 4;          // full[S], empty[S], acc_full[2], acc_empty[2]
+    static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // 7 int32[BN] arrays of per-channel constants
+    static constexpr int OFF_BAR = OFF_CONST + 7 * BN * 4;           // full[S], empty[S], acc_full[2], acc_empty[2]
     static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 4) * 8;  // tensor-memory base, stop flag
     static constexpr int TOTAL = OFF_MISC + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;                   // slack to align the base to 1024 bytes
@@ -96,17 +96,30 @@ __device__ __forceinline__ void epilogue_chunk(const int32_t (&v)[32], const int
     }
 }
 
-// Same chunk in the shift-32 form: one 16-byte constant load, at most one max, one widening multiply-add per output.
+// Same chunk in the shift-32 form with constants from shared memory: half a 16-byte load, one add, at most one
+// max and one widening multiply-add per output.
 template <bool RELU>
-__device__ __forceinline__ void epilogue_chunk_shift32(const int32_t (&v)[32], const int4* s_k, int c0, uint32_t (&out)[8]) {
+__device__ __forceinline__ void epilogue_chunk_shift32(const int32_t (&v)[32], const int32_t* s_bias, const int32_t* s_m2,
+                                                       int c0, uint32_t (&out)[8]) {
 #pragma unroll
     for (int j = 0; j < 8; j++) {
-        const int32_t r0 = requant_shift32<RELU>(v[4 * j + 0], s_k[c0 + 4 * j + 0]);
-        const int32_t r1 = requant_shift32<RELU>(v[4 * j + 1], s_k[c0 + 4 * j + 1]);
-        const int32_t r2 = requant_shift32<RELU>(v[4 * j + 2], s_k[c0 + 4 * j + 2]);
-        const int32_t r3 = requant_shift32<RELU>(v[4 * j + 3], s_k[c0 + 4 * j + 3]);
-        out[j] = pack_sat4(r0, r1, r2, r3);
+        const int4 bi = *reinterpret_cast<const int4*>(s_bias + c0 + 4 * j);
+        const int4 m2 = *reinterpret_cast<const int4*>(s_m2 + c0 + 4 * j);
+        out[j] = pack_sat4(requant_shift32<RELU>(v[4 * j + 0], bi.x, m2.x), requant_shift32<RELU>(v[4 * j + 1], bi.y, m2.y),
+                           requant_shift32<RELU>(v[4 * j + 2], bi.z, m2.z), requant_shift32<RELU>(v[4 * j + 3], bi.w, m2.w));
     }
+}
+
+// The same with the 32 columns' constants already in registers (tiles whose warps keep a fixed column range).
+template <bool RELU>
+__device__ __forceinline__ void epilogue_chunk_shift32_regs(const int32_t (&v)[32], const int32_t (&rb)[32], const int32_t (&rm)[32],
+                                                            uint32_t (&out)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; j++)
+        out[j] = pack_sat4(requant_shift32<RELU>(v[4 * j + 0], rb[4 * j + 0], rm[4 * j + 0]),
+                           requant_shift32<RELU>(v[4 * j + 1], rb[4 * j + 1], rm[4 * j + 1]),
+                           requant_shift32<RELU>(v[4 * j + 2], rb[4 * j + 2], rm[4 * j + 2]),
+                           requant_shift32<RELU>(v[4 * j + 3], rb[4 * j + 3], rm[4 * j + 3]));
 }
 
 // Store one thread's 32 output bytes (columns n .. n+31 of one row).
@@ -139,8 +152,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const uint32_t sbase = raw + pad;
 
     const uint32_t sA = sbase + L::OFF_A, sB = sbase + L::OFF_B;
-    int4* s_k32 = reinterpret_cast<int4*>(smem + L::OFF_CONST);
-    int32_t* s_bias = reinterpret_cast<int32_t*>(smem + L::OFF_CONST) + 4 * BN;
+    int32_t* s_m2 = reinterpret_cast<int32_t*>(smem + L::OFF_CONST);
+    int32_t* s_bias = s_m2 + BN;
     int32_t* s_lo = s_bias + BN;
     int32_t* s_hi = s_lo + BN;
     int32_t* s_mult = s_hi + BN;
@@ -294,6 +307,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int cgroup = (warp - 2) >> 2;             // which share of the columns this warp handles
         int ab = 0, cached_n_blk = -1;
         bool shift32 = false;                           // every channel of the cached block admits the shift-32 form
+        constexpr bool ONE_CHUNK = COLS_PER_GROUP == 32;
+        int32_t rb[ONE_CHUNK ? 32 : 1], rm[ONE_CHUNK ? 32 : 1];   // register copy of the constants (ONE_CHUNK only)
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < sched.num_tiles; tile += gridDim.x) {
             int m_blk, n_blk;
@@ -316,12 +331,17 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const ChanConst cc = make_chan_const(mult, shift, p.relu);
                     s_bias[c] = bias; s_lo[c] = cc.lo; s_hi[c] = cc.hi;
                     s_mult[c] = cc.mult; s_shift[c] = cc.shift; s_rnd[c] = cc.rnd;
-                    int4 k32;
-                    all32 = make_shift32_const(bias, mult, shift, p.relu, k32) && all32;
-                    s_k32[c] = k32;
+                    int32_t m2;
+                    all32 = make_shift32_mult(mult, shift, m2) && all32;
+                    s_m2[c] = m2;
                 }
                 cached_n_blk = n_blk;
                 shift32 = named_barrier_and(2, EPI_THREADS, all32);
+                if constexpr (ONE_CHUNK) if (shift32) {
+                    // this warp's 32 columns are the same for every tile of the block column: keep them in registers
+#pragma unroll
+                    for (int j = 0; j < 32; j++) { rb[j] = s_bias[cgroup * 32 + j]; rm[j] = s_m2[cgroup * 32 + j]; }
+                }
             }
             const int row = m_blk * BM + quarter * 32 + lane;
             int8_t* crow = p.C + (int64_t)row * p.ldc;
@@ -336,8 +356,13 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 tmem_ld_wait();
                 uint32_t out[8];
                 if (shift32) {
-                    if (p.relu) epilogue_chunk_shift32<true>(v, s_k32, c0, out);
-                    else epilogue_chunk_shift32<false>(v, s_k32, c0, out);
+                    if constexpr (ONE_CHUNK) {
+                        if (p.relu) epilogue_chunk_shift32_regs<true>(v, rb, rm, out);
+                        else epilogue_chunk_shift32_regs<false>(v, rb, rm, out);
+                    } else {
+                        if (p.relu) epilogue_chunk_shift32<true>(v, s_bias, s_m2, c0, out);
+                        else epilogue_chunk_shift32<false>(v, s_bias, s_m2, c0, out);
+                    }
                 } else {
                     epilogue_chunk(v, s_bias, s_lo, s_hi, s_mult, s_shift, s_rnd, c0, out);
                 }
