@@ -193,6 +193,8 @@ static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_
     if (rc) return rc;
     KLoop kl{};
     kl.cb = BK; kl.nsub = 1; kl.num_kblocks = (K + BK - 1) / BK;
+    kl.num_iters = kl.num_kblocks;
+    kl.mmas_last = ((K - (kl.num_iters - 1) * BK) + 31) / 32;
     return run_tc(ctx, false, tmA, kl, bn, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
 }
 
@@ -218,6 +220,8 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     KLoop kl{};
     kl.cb = cb; kl.nsub = BK / cb; kl.cblocks = C / cb; kl.num_kblocks = R * S * kl.cblocks;
     kl.P = P; kl.Q = Q; kl.S = S;
+    kl.num_iters = (kl.num_kblocks + kl.nsub - 1) / kl.nsub;
+    kl.mmas_last = (kl.num_kblocks - (kl.num_iters - 1) * kl.nsub) * (cb / 32);
     kl.stride_h = stride_h; kl.stride_w = stride_w; kl.pad_h = pad_h; kl.pad_w = pad_w;
     const int K = R * S * C;
     return run_tc(ctx, true, tmA, kl, bn, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);

@@ -30,6 +30,8 @@ constexpr int UMMA_K = 32;       // K per tcgen05.mma for 8-bit operands
 // Convolution: cb = channel block, nsub = 128 / cb, num_kblocks = R * S * (C / cb).
 struct KLoop {
     int cb, nsub, num_kblocks;
+    int num_iters;                        // ring slots per tile = ceil(num_kblocks / nsub)
+    int mmas_last;                        // tcgen05.mma instructions of a tile's last slot (1..4)
     int P, Q, S, cblocks;                 // convolution only: output extent, filter width, C / cb
     int stride_h, stride_w, pad_h, pad_w;
 };
@@ -37,6 +39,7 @@ struct KLoop {
 struct TileSched {
     int m_tiles, n_tiles, num_tiles, group_m;
     __device__ __forceinline__ void map(int tile, int& m_blk, int& n_blk) const {
+        if (n_tiles == 1) { m_blk = tile; n_blk = 0; return; }   // one block column: no divisions
         const int width = group_m * n_tiles;
         const int g = tile / width;
         const int first_m = g * group_m;
@@ -256,46 +259,51 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // K-major operands: rows cb bytes apart, swizzled over cb bytes, 8-row groups 8*cb bytes apart;
         // a 32-byte step along K inside a swizzle row is a plain address offset.
         const uint64_t swz = kl.cb == 128 ? SWZ_128B : (kl.cb == 64 ? SWZ_64B : SWZ_32B);
-        const uint32_t sbo = 8 * kl.cb;
-        const uint64_t desc_hi = make_smem_desc(0, 16, sbo, swz);   // everything but the start address
+        const uint64_t desc_hi = make_smem_desc(0, 16, 8 * kl.cb, swz);   // everything but the start address
+        const bool leader = elect_one();
+        // A full ring slot always takes BK / 32 = 4 instructions; their operand offsets (in 16-byte descriptor
+        // units) inside the slot depend only on the sub-block geometry.
+        const int per_sub = kl.cb / UMMA_K;
+        uint32_t offA[4], offB[4];
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            const int sub = i / per_sub, k = i - sub * per_sub;
+            offA[i] = (sub * a_sub_bytes + k * UMMA_K) >> 4;
+            offB[i] = (sub * b_sub_bytes + k * UMMA_K) >> 4;
+        }
+        const uint32_t a_base = (sA & 0x3FFFFu) >> 4, b_base = (sB & 0x3FFFFu) >> 4;
         int stage = 0, ab = 0;
         uint32_t phase = 0, acc_phase = 0;
+        bool ready = false;                              // the slot (stage, phase) is already known to be full
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
             if (!mbar_wait_warp(bar_acc_empty + 8 * ab, acc_phase ^ 1, env, DEV_TIMEOUT_MMA_ACC)) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + ab * BN;
-            uint32_t accumulate = 0;
-            for (int kbi = 0; kbi < kl.num_kblocks;) {
-                if (!mbar_wait_warp(bar_full + 8 * stage, phase, env, DEV_TIMEOUT_MMA_FULL)) { ok = false; break; }
+            for (int it = 0; it < kl.num_iters; it++) {
+                if (!ready && !mbar_wait_warp(bar_full + 8 * stage, phase, env, DEV_TIMEOUT_MMA_FULL)) { ok = false; break; }
                 tc_fence_after();
-                const int nb = min(kl.nsub, kl.num_kblocks - kbi);
-                const bool leader = elect_one();
-                for (int j = 0; j < nb; j++, kbi++) {
-                    const uint32_t a0 = sA + stage * L::A_BYTES + j * a_sub_bytes;
-                    const uint32_t b0 = sB + stage * L::B_BYTES + j * b_sub_bytes;
-                    int ksteps = kl.cb / UMMA_K;
-                    if (!CONV) {                       // GEMM: the last block may be ragged in K
-                        const int rem = p.K - kbi * BK;
-                        if (rem < BK) ksteps = (rem + UMMA_K - 1) / UMMA_K;
-                    }
-                    if (leader) {
-                        for (int k = 0; k < ksteps; k++) {
-                            const uint64_t ad = desc_hi | (uint64_t)(((a0 + k * UMMA_K) & 0x3FFFFu) >> 4);
-                            const uint64_t bd = desc_hi | (uint64_t)(((b0 + k * UMMA_K) & 0x3FFFFu) >> 4);
-                            mma_i8_ss(d_tmem, ad, bd, idesc, accumulate);
-                            accumulate = 1;
-                        }
-                    }
-                    accumulate = 1;
+                // poll the next slot now; its answer is only needed after this slot's instructions are issued
+                int nstage = stage + 1;
+                uint32_t nphase = phase;
+                if (nstage == STAGES) { nstage = 0; nphase ^= 1; }
+                const bool peek = mbar_test_wait(bar_full + 8 * nstage, nphase);
+                if (leader) {
+                    const int nm = it == kl.num_iters - 1 ? kl.mmas_last : 4;
+                    const uint32_t a0 = a_base + stage * (L::A_BYTES >> 4), b0 = b_base + stage * (L::B_BYTES >> 4);
+#pragma unroll
+                    for (int i = 0; i < 4; i++)
+                        if (i < nm)
+                            mma_i8_ss(d_tmem, desc_hi | (uint64_t)(a0 + offA[i]), desc_hi | (uint64_t)(b0 + offB[i]), idesc,
+                                      (it | i) != 0 ? 1u : 0u);
+                    tc_commit(bar_empty + 8 * stage);    // slot reusable once these MMAs have read it
                 }
-                if (leader) tc_commit(bar_empty + 8 * stage);   // slot reusable once these MMAs have read it
-                __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                ready = __all_sync(0xffffffffu, peek);
+                stage = nstage;
+                phase = nphase;
             }
             if (!ok) break;
-            if (elect_one()) tc_commit(bar_acc_full + 8 * ab);  // accumulator complete
-            __syncwarp();
+            if (leader) tc_commit(bar_acc_full + 8 * ab);   // accumulator complete
             ab ^= 1;
             if (ab == 0) acc_phase ^= 1;
         }
