@@ -143,6 +143,7 @@ __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmTcParams p) {
     using L = TcSmem<BN, STAGES>;
     constexpr int EPI_THREADS = 32 * EPI_WARPS;
+    constexpr int NTHREADS = 64 + EPI_THREADS;
     constexpr int COL_GROUPS = EPI_WARPS / 4;          // warps sharing a lane quarter split the columns
     constexpr int COLS_PER_GROUP = BN / COL_GROUPS;
     static_assert(EPI_WARPS == 4 || EPI_WARPS == 8, "4 or 8 epilogue warps");
@@ -194,10 +195,18 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *s_tmem, 0);   // same value in every lane, known uniform
+    // Set-up barrier.  The producer warp initialised the mbarriers itself and needs nothing from the others, so it
+    // only signals and starts loading at once; everybody else waits for the barriers and the tensor-memory address.
+    uint32_t tmem_base = 0;
+    if (warp == 0) {
+        __syncwarp();
+        named_barrier_arrive(15, NTHREADS);
+    } else {
+        tc_fence_before();
+        named_barrier(15, NTHREADS);
+        tc_fence_after();
+        tmem_base = __shfl_sync(0xffffffffu, *s_tmem, 0);   // same value in every lane, known uniform
+    }
 
     const TileSched sched = p.sched;
     const KLoop kl = p.kl;
@@ -318,15 +327,14 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         constexpr bool ONE_CHUNK = COLS_PER_GROUP == 32;
         int32_t rb[ONE_CHUNK ? 32 : 1], rm[ONE_CHUNK ? 32 : 1];   // register copy of the constants (ONE_CHUNK only)
         uint32_t acc_phase = 0;
+        bool dead = false;
         for (int tile = blockIdx.x; tile < sched.num_tiles; tile += gridDim.x) {
             int m_blk, n_blk;
             sched.map(tile, m_blk, n_blk);
-            bool ok = mbar_wait(bar_acc_full + 8 * ab, acc_phase, env, DEV_TIMEOUT_EPILOGUE);
-            ok = named_barrier_and(1, EPI_THREADS, ok);   // all agree; also: previous tile's constants are no longer read
-            if (!ok) break;
-            tc_fence_after();
             const int n0 = n_blk * BN;
             if (n_blk != cached_n_blk) {
+                // new block column: rebuild the per-channel constants (before waiting, so this overlaps the main loop)
+                named_barrier(1, EPI_THREADS);            // nobody still reads the previous column's constants
                 bool all32 = true;
                 for (int c = etid; c < BN; c += EPI_THREADS) {
                     const int n = n0 + c;
@@ -351,6 +359,11 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     for (int j = 0; j < 32; j++) { rb[j] = s_bias[cgroup * 32 + j]; rm[j] = s_m2[cgroup * 32 + j]; }
                 }
             }
+            // A warp whose wait expired stays in the loop without touching the accumulators, so that the barriers
+            // above still see every warp; the stop flag it raised ends the other roles.
+            if (!dead) dead = !__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * ab, acc_phase, env, DEV_TIMEOUT_EPILOGUE));
+            if (dead) continue;
+            tc_fence_after();
             const int row = m_blk * BM + quarter * 32 + lane;
             int8_t* crow = p.C + (int64_t)row * p.ldc;
             const uint32_t t0 = tmem_base + ab * BN + ((uint32_t)(quarter * 32) << 16);

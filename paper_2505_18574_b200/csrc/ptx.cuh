@@ -144,6 +144,10 @@ __device__ __forceinline__ bool named_barrier_and(int id, int nthreads, bool pre
         : "memory");
     return out != 0;
 }
+// Arrive without waiting (counts toward the same barrier as the threads that call named_barrier on it).
+__device__ __forceinline__ void named_barrier_arrive(int id, int nthreads) {
+    asm volatile("barrier.cta.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 __device__ __forceinline__ void named_barrier(int id, int nthreads) {
     asm volatile("barrier.cta.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
