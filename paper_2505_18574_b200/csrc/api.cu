@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <mutex>
+#include <utility>
 
 #include "../../include/i8ops.h"
 #include "batched_tc.cuh"
@@ -33,6 +34,7 @@ static DeviceCtx g_ctx[MAX_DEVICES];
 static std::mutex g_mutex;
 static int g_path_mode = 0;                      // 0 auto, 1 generic only, 2 tensor whenever legal
 static uint64_t g_wait_limit_ns = 2000ull * 1000 * 1000;
+static int g_pdl = 1;                            // programmatic dependent launch (I8OPS_PDL=0 turns it off)
 static int g_force_bn = -1;                      // tuning override from the environment (I8OPS_FORCE_BN)
 
 static thread_local int t_last_path = I8_PATH_NONE;
@@ -82,6 +84,8 @@ static int get_ctx(DeviceCtx** out) {
         }
         const char* bn = getenv("I8OPS_FORCE_BN");
         if (bn) g_force_bn = atoi(bn);
+        const char* pdl = getenv("I8OPS_PDL");
+        if (pdl) g_pdl = atoi(pdl);
         c.ready = true;
     }
     *out = &c;
@@ -102,6 +106,24 @@ static int make_tmap(CUtensorMap* tm, const void* base, int rank, const uint64_t
     return I8_OK;
 }
 
+// Launch on `st`; with programmatic stream serialisation the kernel may be scheduled while its predecessor in
+// the stream drains (the kernels wait for their dependencies before touching global memory).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_kernel(void (*kern)(KArgs...), bool overlap, int grid, int block, size_t smem, cudaStream_t st,
+                                 Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (g_pdl && overlap) ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ------------------------------------------------------------------------------------------------ launches
@@ -119,14 +141,16 @@ static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUt
         ctx->attr_set[slot] = true;
     }
     const int grid = p.sched.num_tiles < ctx->sm_count ? p.sched.num_tiles : ctx->sm_count;
-    kern<<<grid, 64 + 32 * EPI_WARPS, L::DYN_BYTES, st>>>(tmA, tmB, p);
-    CUDA_TRY(cudaGetLastError());
+    // short kernels gain from overlapping their launch with the predecessor's tail; long ones do not need it
+    const bool overlap = 2.0 * p.M * p.N * p.K < 4e10;
+    CUDA_TRY(launch_kernel(kern, overlap, grid, 64 + 32 * EPI_WARPS, L::DYN_BYTES, st, tmA, tmB, p));
     return I8_OK;
 }
 
-// Tile width: model each K block as operand-delivery bound (256 + 2*BN cycles) and pick the width with the
-// fewest total cycles over all waves; ties go to the wider tile.
-static int choose_bn(int M, int N, int sm_count) {
+// Tile width.  Cost model in SM cycles: every wave of tiles pays, per 128-byte K block, an operand-delivery
+// bound of 256 + 2*BN, plus a fixed 400 per tile; the last tile's read-out (about 14 cycles per column) is
+// exposed.  The width with the lowest total wins; ties go to the wider tile.
+static int choose_bn(int M, int N, int num_kb, int sm_count) {
     if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256) return g_force_bn;
     const int cands[3] = {256, 128, 64};
     int best = 64;
@@ -137,7 +161,7 @@ static int choose_bn(int M, int N, int sm_count) {
         if (bn > 64 && bn - 64 >= ((N + 63) / 64) * 64) continue;   // tile mostly empty
         const int64_t tiles = (int64_t)m_tiles * ((N + bn - 1) / bn);
         const int64_t waves = (tiles + sm_count - 1) / sm_count;
-        const double cost = (double)waves * (256.0 + 2.0 * bn);
+        const double cost = (double)waves * ((double)num_kb * (256.0 + 2.0 * bn) + 400.0) + 14.0 * bn;
         if (cost < best_cost - 1e-9) { best_cost = cost; best = bn; }
     }
     return best;
@@ -184,7 +208,7 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
 static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
                        int K, int relu, cudaStream_t st) {
-    const int bn = choose_bn(M, N, ctx->sm_count);
+    const int bn = choose_bn(M, N, (K + BK - 1) / BK, ctx->sm_count);
     CUtensorMap tmA;
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
     const uint64_t str[1] = {(uint64_t)lda};
@@ -204,7 +228,7 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
                        int stride_h, int stride_w, int pad_h, int pad_w, int relu, cudaStream_t st) {
     const int cb = C % 128 == 0 ? 128 : (C % 64 == 0 ? 64 : 32);
     const int M = N * P * Q;
-    const int bn = choose_bn(M, Kf, ctx->sm_count);
+    const int bn = choose_bn(M, Kf, (R * S * C + BK - 1) / BK, ctx->sm_count);
     CUtensorMap tmA;
     {
         const cuuint64_t gdim[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
@@ -261,8 +285,7 @@ static int run_batched_pair(DeviceCtx* ctx, const int8_t* A, int64_t a_rs, int64
     }
     const int pairs = (batch + 1) / 2;
     const int grid = pairs < ctx->sm_count ? pairs : ctx->sm_count;
-    batched_pair_i8_kernel<<<grid, PAIR_THREADS, PairSmem::DYN_BYTES, st>>>(tmA, tmB, p);
-    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(launch_kernel(batched_pair_i8_kernel, true, grid, PAIR_THREADS, PairSmem::DYN_BYTES, st, tmA, tmB, p));
     return I8_OK;
 }
 

@@ -148,6 +148,8 @@ batched_pair_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
     }
+    grid_launch_dependents();
+    grid_dependency_wait();   // global memory is touched from here on
     // per-channel constants of the 64 output columns (shared by every problem of the batch)
     bool my32 = true;
     if (threadIdx.x < 64) {

@@ -195,6 +195,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
     }
+    // Everything above touched only shared and tensor memory; from here on global memory is read and written.
+    grid_launch_dependents();
+    grid_dependency_wait();
     // Set-up barrier.  The producer warp initialised the mbarriers itself and needs nothing from the others, so it
     // only signals and starts loading at once; everybody else waits for the barriers and the tensor-memory address.
     uint32_t tmem_base = 0;
