@@ -189,6 +189,11 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
     p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
     p.sched.group_m = 16;
     p.kl = kl;
+    {
+        // resident B: one block column, and all of B's K blocks fit the ring's B region
+        const int stages = bn == 256 ? 4 : (bn == 128 ? 6 : 8);
+        p.kl.b_resident = (p.sched.n_tiles == 1 && (int64_t)kl.num_kblocks * bn * kl.cb <= (int64_t)stages * bn * BK) ? 1 : 0;
+    }
     p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);   // SM clock stays below 2 GHz: at least the asked time
     p.dev_status = ctx->dev_status;
     if (conv) {
@@ -244,6 +249,8 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     KLoop kl{};
     kl.cb = cb; kl.nsub = BK / cb; kl.cblocks = C / cb; kl.num_kblocks = R * S * kl.cblocks;
     kl.P = P; kl.Q = Q; kl.S = S;
+    kl.inv_pq = P * Q == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)(P * Q));
+    kl.inv_q = Q == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)Q);
     kl.num_iters = (kl.num_kblocks + kl.nsub - 1) / kl.nsub;
     kl.mmas_last = (kl.num_kblocks - (kl.num_iters - 1) * kl.nsub) * (cb / 32);
     kl.stride_h = stride_h; kl.stride_w = stride_w; kl.pad_h = pad_h; kl.pad_w = pad_w;

@@ -34,7 +34,16 @@ struct KLoop {
     int mmas_last;                        // tcgen05.mma instructions of a tile's last slot (1..4)
     int P, Q, S, cblocks;                 // convolution only: output extent, filter width, C / cb
     int stride_h, stride_w, pad_h, pad_w;
+    uint32_t inv_pq, inv_q;               // floor(2^32 / (P*Q)) and floor(2^32 / Q) (0xffffffff for a divisor of 1)
+    int b_resident;                       // the whole B operand of the (single) block column stays in shared memory
 };
+
+// n / d for n < 2^31 with inv = floor(2^32 / d): the estimate is at most one too small.
+__device__ __forceinline__ int fast_div(int n, int d, uint32_t inv) {
+    int q = (int)__umulhi((uint32_t)n, inv);
+    if (n - q * d >= d) ++q;
+    return q;
+}
 
 struct TileSched {
     int m_tiles, n_tiles, num_tiles, group_m;
@@ -72,8 +81,8 @@ struct TcSmem {
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
     static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // 7 int32[BN] arrays of per-channel constants
-    static constexpr int OFF_BAR = OFF_CONST + 7 * BN * 4;           // full[S], empty[S], acc_full[2], acc_empty[2]
-    static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 4) * 8;  // tensor-memory base, stop flag
+    static constexpr int OFF_BAR = OFF_CONST + 7 * BN * 4;           // full[S], empty[S], acc_full[2], acc_empty[2], b_resident
+    static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 5) * 8;  // tensor-memory base, stop flag
     static constexpr int TOTAL = OFF_MISC + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;                   // slack to align the base to 1024 bytes
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // BN in {64,128,256}: a power of two
@@ -167,6 +176,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const uint32_t bar_empty = bar_full + STAGES * 8;
     const uint32_t bar_acc_full = bar_empty + STAGES * 8;
     const uint32_t bar_acc_empty = bar_acc_full + 2 * 8;
+    const uint32_t bar_bres = bar_acc_empty + 2 * 8;
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC);
     volatile int* s_stop = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
 
@@ -184,6 +194,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             mbar_init(bar_acc_full + 8 * b, 1);
             mbar_init(bar_acc_empty + 8 * b, EPI_THREADS);
         }
+        mbar_init(bar_bres, 1);
         *s_stop = 0;
         fence_barrier_init();
     }
@@ -220,6 +231,15 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int stage = 0;
         uint32_t phase = 0, issued = 0, issued_phase = 0;
         bool ok = true;
+        const bool leader = elect_one();
+        const bool bres = kl.b_resident != 0;
+        if (bres && blockIdx.x < sched.num_tiles && leader) {
+            // the paper's "keep B resident" step: the whole (small) B operand is fetched once per CTA into the
+            // region the ring would otherwise use for B, and only A streams
+            mbar_expect_tx(bar_bres, kl.num_kblocks * b_sub_bytes);
+            for (int kb = 0; kb < kl.num_kblocks; kb++) tma_load_2d(sB + kb * b_sub_bytes, &tmB, bar_bres, kb * kl.cb, 0);
+        }
+        const uint32_t stage_tx = a_sub_bytes + (bres ? 0u : b_sub_bytes);
         for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
             int m_blk, n_blk;
             sched.map(tile, m_blk, n_blk);
@@ -228,9 +248,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 // first output pixel of the tile -> position of filter tap (0,0) in the input image
                 const int m0 = m_blk * BM;
                 const int pq = kl.P * kl.Q;
-                img = m0 / pq;
+                img = fast_div(m0, pq, kl.inv_pq);
                 const int rem = m0 - img * pq;
-                const int op = rem / kl.Q, oq = rem - op * kl.Q;
+                const int op = fast_div(rem, kl.Q, kl.inv_q), oq = rem - op * kl.Q;
                 h0 = op * kl.stride_h - kl.pad_h;
                 w0 = oq * kl.stride_w - kl.pad_w;
             }
@@ -239,8 +259,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                 const int nb = min(kl.nsub, kl.num_kblocks - kbi);
                 const uint32_t full = bar_full + 8 * stage;
-                const bool leader = elect_one();
-                if (leader) mbar_expect_tx(full, nb * (a_sub_bytes + b_sub_bytes));
+                if (leader) mbar_expect_tx(full, nb * stage_tx);
                 for (int j = 0; j < nb; j++, kbi++) {
                     const uint32_t dstA = sA + stage * L::A_BYTES + j * a_sub_bytes;
                     const uint32_t dstB = sB + stage * L::B_BYTES + j * b_sub_bytes;
@@ -250,7 +269,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     } else {
                         if (leader) tma_load_2d(dstA, &tmA, full, kbi * BK, m_blk * BM);
                     }
-                    if (leader) tma_load_2d(dstB, &tmB, full, kbi * kl.cb, n_blk * BN);
+                    if (leader && !bres) tma_load_2d(dstB, &tmB, full, kbi * kl.cb, n_blk * BN);
                 }
                 issued |= 1u << stage;
                 issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
@@ -259,6 +278,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
         if (*s_stop) {
             // stopping early: let every copy this warp started land before the CTA retires
+            if (bres && blockIdx.x < sched.num_tiles && !mbar_wait_drain(bar_bres, 0, p.wait_limit_cycles))
+                atomicCAS(p.dev_status, 0u, (unsigned)DEV_TIMEOUT_DRAIN);
             for (int s = 0; s < STAGES; s++)
                 if (issued & (1u << s))
                     if (!mbar_wait_drain(bar_full + 8 * s, (issued_phase >> s) & 1u, p.wait_limit_cycles))
@@ -288,6 +309,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         uint32_t phase = 0, acc_phase = 0;
         bool ready = false;                              // the slot (stage, phase) is already known to be full
         bool ok = true;
+        const bool bres = kl.b_resident != 0;
+        const uint32_t b_iter_units = (kl.nsub * b_sub_bytes) >> 4;   // resident B: descriptor units per ring slot's worth of K
+        if (bres && blockIdx.x < sched.num_tiles) ok = mbar_wait_warp(bar_bres, 0, env, DEV_TIMEOUT_MMA_FULL);
         for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
             if (!mbar_wait_warp(bar_acc_empty + 8 * ab, acc_phase ^ 1, env, DEV_TIMEOUT_MMA_ACC)) break;
             tc_fence_after();
@@ -302,7 +326,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 const bool peek = mbar_test_wait(bar_full + 8 * nstage, nphase);
                 if (leader) {
                     const int nm = it == kl.num_iters - 1 ? kl.mmas_last : 4;
-                    const uint32_t a0 = a_base + stage * (L::A_BYTES >> 4), b0 = b_base + stage * (L::B_BYTES >> 4);
+                    const uint32_t a0 = a_base + stage * (L::A_BYTES >> 4);
+                    const uint32_t b0 = b_base + (bres ? it * b_iter_units : stage * (L::B_BYTES >> 4));
 #pragma unroll
                     for (int i = 0; i < 4; i++)
                         if (i < nm)
