@@ -4,12 +4,14 @@
 One "step" runs the three large GEMMs of the headline workload (4096^3, 8192^3, 16384x4096x8192; per-output-
 channel requantisation, ReLU off) once each through the C-ABI library, on synthetic seeded inputs.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--details]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-details]
 
 prints ONE JSON line.  `value` is int8 TOPS (2*MACs / time) summed over all ranks with operands resident in
 HBM; `e2e` is the same metric through the host-buffer entry point with the copies inside the timed region;
 `roofline` is the tensor kernel's achieved rate against the measured peak; `cpu_baseline` is the CPU oracle
-on a bounded sample of the same workload.  `--impl reference` times the oracle alone (rank 0 only).
+on a bounded sample of the same workload; `details` lists every other configuration (256^3, the convolutions, the
+tall-skinny and batched products) timed one by one after the headline measurement.  `--impl reference` times the
+oracle alone (rank 0 only).
 """
 from __future__ import annotations
 
@@ -181,7 +183,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--details", action="store_true", help="add per-problem timings of every workload configuration")
+    ap.add_argument("--no-details", action="store_true", help="skip the per-problem timings of the other workload configurations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -312,7 +314,7 @@ def main():
     e2e_exact = all(np.array_equal(host[j]["C"].numpy(), dev_t[j]["C"].cpu().numpy()) for j in range(3))
 
     details = None
-    if args.details and rank == 0:
+    if not args.no_details and rank == 0 and world == 1:
         from paper_2505_18574_b200 import bench_details
         pk = measured_peaks()
         details = bench_details.run(dev, peak_tops=2 * pk["bf16_burst"], peak_gbs=pk["hbm_gbs"])
