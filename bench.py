@@ -213,8 +213,10 @@ def main():
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    from paper_2505_18574_b200 import sharding
     if rank != 0:                       # independent problems per rank: same shapes, different draws
-        problems = [inputs.make_gemm(p.M, p.N, p.K, p.seed + 1000 * rank, per_channel=1, relu=0, name=p.name) for p in problems]
+        problems = [inputs.make_gemm(p.M, p.N, p.K, sharding.rank_seed(p.seed, rank), per_channel=1, relu=0, name=p.name)
+                    for p in problems]
 
     dev_t = []
     for p in problems:
@@ -277,12 +279,9 @@ def main():
     per_problem_ms = [t / args.steps for t in per_problem_ms]
     assert i8.last_device_status() == 0
 
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max = float(t.item())
+    total_ms_max = sharding.max_over_ranks(total_ms, dev)
     ops_step = sum(gemm_ops(p) for p in problems)
-    value = world * ops_step * args.steps / (total_ms_max * 1e-3) / 1e12
+    value = sharding.whole_job_rate(ops_step * args.steps, world, total_ms_max) / 1e12
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     host = []
@@ -305,10 +304,7 @@ def main():
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_value = world * ops_step * args.e2e_steps / (float(t.item()) * 1e-3) / 1e12
+    e2e_value = sharding.whole_job_rate(ops_step * args.e2e_steps, world, sharding.max_over_ranks(e2e_ms, dev)) / 1e12
     h2d = sum(p.M * p.K + p.N * p.K + 4 * p.N * 3 for p in problems)
     d2h = sum(p.M * p.N for p in problems)
     e2e_exact = all(np.array_equal(host[j]["C"].numpy(), dev_t[j]["C"].cpu().numpy()) for j in range(3))
