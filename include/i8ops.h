@@ -132,6 +132,11 @@ const char* i8_status_string(int status);
  * this library on the current device since the last call, or I8_ERR_CUDA.  Clears the record. */
 int i8ops_last_device_status(void* stream);
 
+/* Self-test of the failure path (no counterpart in the paper): launches one small CTA that waits, for at most
+ * `limit_ms` (1..1000) milliseconds, on a barrier that nothing signals.  The kernel returns by itself and the next
+ * i8ops_last_device_status() reports I8_ERR_TIMEOUT.  Nothing faults, traps or hangs. */
+int i8ops_selftest_bounded_wait(int limit_ms, void* stream);
+
 /* cudaError_t of the most recent failed CUDA call made by this library on this thread (0 if none). */
 int i8ops_last_cuda_error(void);
 

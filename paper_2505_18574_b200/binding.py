@@ -29,6 +29,7 @@ SIGNATURES = {
     "gemm_i8_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
     "i8_status_string": (ctypes.c_char_p, [_int]),
     "i8ops_last_device_status": (_int, [_vp]),
+    "i8ops_selftest_bounded_wait": (_int, [_int, _vp]),
     "i8ops_last_cuda_error": (_int, []),
     "i8ops_last_path": (_int, []),
     "i8ops_set_path": (_int, [_int]),

@@ -505,6 +505,17 @@ int i8ops_last_device_status(void* stream) {
     return I8_OK;
 }
 
+int i8ops_selftest_bounded_wait(int limit_ms, void* stream) {
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    if (limit_ms < 1) limit_ms = 1;
+    if (limit_ms > 1000) limit_ms = 1000;
+    bounded_wait_selftest_kernel<<<1, 64, 0, (cudaStream_t)stream>>>((long long)limit_ms * 2000000ll, ctx->dev_status);
+    CUDA_TRY(cudaGetLastError());
+    return I8_OK;
+}
+
 int i8ops_last_cuda_error(void) { return t_last_cuda; }
 int i8ops_last_path(void) { return t_last_path; }
 

@@ -3,6 +3,7 @@
 // combinations, K == 0) and tiny problems, and double as an in-library cross-check of the tensor paths.
 #pragma once
 #include "epilogue.cuh"
+#include "ptx.cuh"
 
 namespace i8 {
 
@@ -63,6 +64,24 @@ __global__ void __launch_bounds__(256) conv2d_i8_generic_kernel(const GenericCon
         const int ci = p.per_channel ? k : 0;
         p.y[idx] = (int8_t)requant_wide(acc, p.bias ? p.bias[k] : 0, p.relu, p.mult[ci], p.shift[ci]);
     }
+}
+
+// Self-test of the bounded wait: one CTA waits on an mbarrier that nothing ever signals.  The wait must give
+// up after `limit_cycles`, record DEV_TIMEOUT_TEST in the status word and return normally.
+__global__ void bounded_wait_selftest_kernel(long long limit_cycles, unsigned* dev_status) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int stop;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        stop = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    const WaitEnv env{&stop, dev_status, limit_cycles};
+    mbar_wait_warp(b, 0, env, DEV_TIMEOUT_TEST);
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_inval(b);
 }
 
 }  // namespace i8

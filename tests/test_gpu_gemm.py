@@ -136,3 +136,18 @@ def test_config4a_tall_skinny():
     want = H.gemm_oracle(p)
     H.assert_same(got, want, p.name)
     H.not_degenerate(want)
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A wait that nothing satisfies must end by itself with a status the host can read; the next call still works."""
+    import time
+    import paper_2505_18574_b200 as i8
+    L = i8.lib()
+    assert i8.last_device_status() == 0
+    t0 = time.time()
+    assert L.i8ops_selftest_bounded_wait(20, None) == 0
+    assert i8.last_device_status() == 8            # I8_ERR_TIMEOUT
+    assert time.time() - t0 < 5.0
+    assert i8.last_device_status() == 0            # the record is cleared by the query
+    p = inputs.make_gemm(128, 64, 64, 3, per_channel=0, relu=1)
+    H.assert_same(H.gemm_gpu(p), H.gemm_oracle(p), "gemm after a timed-out wait")
