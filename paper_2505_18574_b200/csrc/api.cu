@@ -131,11 +131,11 @@ static CUtensorMapSwizzle swizzle_for(int cb) {
     return cb == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (cb == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
 }
 
-template <int BN, int STAGES, bool CONV, int EPI_WARPS>
+template <int BN, int STAGES, bool CONV, int EPI_WARPS, int NPROD>
 static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUtensorMap& tmB, GemmTcParams& p,
                      cudaStream_t st) {
     using L = TcSmem<BN, STAGES>;
-    auto kern = gemm_i8_tc_kernel<BN, STAGES, CONV, EPI_WARPS>;
+    auto kern = gemm_i8_tc_kernel<BN, STAGES, CONV, EPI_WARPS, NPROD>;
     if (!ctx->attr_set[slot]) {
         CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES));
         ctx->attr_set[slot] = true;
@@ -143,7 +143,7 @@ static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUt
     const int grid = p.sched.num_tiles < ctx->sm_count ? p.sched.num_tiles : ctx->sm_count;
     // short kernels gain from overlapping their launch with the predecessor's tail; long ones do not need it
     const bool overlap = 2.0 * p.M * p.N * p.K < 4e10;
-    CUDA_TRY(launch_kernel(kern, overlap, grid, 64 + 32 * EPI_WARPS, L::DYN_BYTES, st, tmA, tmB, p));
+    CUDA_TRY(launch_kernel(kern, overlap, grid, 32 * (1 + NPROD) + 32 * EPI_WARPS, L::DYN_BYTES, st, tmA, tmB, p));
     return I8_OK;
 }
 
@@ -198,15 +198,15 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
     p.dev_status = ctx->dev_status;
     if (conv) {
         switch (bn) {
-            case 256: return launch_tc<256, 4, true, 8>(ctx, 3, tmA, tmB, p, st);
-            case 128: return launch_tc<128, 6, true, 8>(ctx, 4, tmA, tmB, p, st);
-            default:  return launch_tc<64, 8, true, 8>(ctx, 5, tmA, tmB, p, st);
+            case 256: return launch_tc<256, 4, true, 8, 2>(ctx, 3, tmA, tmB, p, st);
+            case 128: return launch_tc<128, 6, true, 8, 2>(ctx, 4, tmA, tmB, p, st);
+            default:  return launch_tc<64, 8, true, 8, 2>(ctx, 5, tmA, tmB, p, st);
         }
     }
     switch (bn) {
-        case 256: return launch_tc<256, 4, false, 4>(ctx, 0, tmA, tmB, p, st);
-        case 128: return launch_tc<128, 6, false, 4>(ctx, 1, tmA, tmB, p, st);
-        default:  return launch_tc<64, 8, false, 8>(ctx, 2, tmA, tmB, p, st);
+        case 256: return launch_tc<256, 4, false, 4, 1>(ctx, 0, tmA, tmB, p, st);
+        case 128: return launch_tc<128, 6, false, 4, 1>(ctx, 1, tmA, tmB, p, st);
+        default:  return launch_tc<64, 8, false, 8, 1>(ctx, 2, tmA, tmB, p, st);
     }
 }
 

@@ -147,12 +147,15 @@ __device__ __forceinline__ void store_row_chunk(int8_t* crow, int n, int N, bool
     }
 }
 
-template <int BN, int STAGES, bool CONV, int EPI_WARPS>
-__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
+template <int BN, int STAGES, bool CONV, int EPI_WARPS, int NPROD>
+__global__ void __launch_bounds__(32 * (1 + NPROD) + 32 * EPI_WARPS, 1)
 gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmTcParams p) {
     using L = TcSmem<BN, STAGES>;
     constexpr int EPI_THREADS = 32 * EPI_WARPS;
-    constexpr int NTHREADS = 64 + EPI_THREADS;
+    constexpr int NTHREADS = 32 * (1 + NPROD) + EPI_THREADS;
+    constexpr int PROD2_WARP = 2 + EPI_WARPS;         // the optional second producer is the last warp
+    static_assert(NPROD == 1 || NPROD == 2, "one or two producer warps");
+    static_assert(STAGES % 2 == 0, "two producers alternate ring slots");
     constexpr int COL_GROUPS = EPI_WARPS / 4;          // warps sharing a lane quarter split the columns
     constexpr int COLS_PER_GROUP = BN / COL_GROUPS;
     static_assert(EPI_WARPS == 4 || EPI_WARPS == 8, "4 or 8 epilogue warps");
@@ -215,6 +218,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (warp == 0) {
         __syncwarp();
         named_barrier_arrive(15, NTHREADS);
+    } else if (NPROD == 2 && warp == PROD2_WARP) {
+        named_barrier(15, NTHREADS);                      // needs the initialised barriers, nothing else
     } else {
         tc_fence_before();
         named_barrier(15, NTHREADS);
@@ -226,14 +231,17 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const KLoop kl = p.kl;
     const uint32_t a_sub_bytes = BM * kl.cb, b_sub_bytes = BN * kl.cb;
 
-    if (warp == 0) {
+    if (warp == 0 || (NPROD == 2 && warp == PROD2_WARP)) {
         // ------------------------------------------------------------------ producer (whole warp loops, one lane issues)
+        // With two producer warps, warp 0 fills the even ring slots and the last warp the odd ones; both walk the
+        // same sequence of tiles and slots and skip the slots that are not theirs.
+        const int pid = warp == 0 ? 0 : 1;
         int stage = 0;
         uint32_t phase = 0, issued = 0, issued_phase = 0;
         bool ok = true;
         const bool leader = elect_one();
         const bool bres = kl.b_resident != 0;
-        if (bres && blockIdx.x < sched.num_tiles && leader) {
+        if (bres && pid == 0 && blockIdx.x < sched.num_tiles && leader) {
             // the paper's "keep B resident" step: the whole (small) B operand is fetched once per CTA into the
             // region the ring would otherwise use for B, and only A streams
             mbar_expect_tx(bar_bres, kl.num_kblocks * b_sub_bytes);
@@ -256,8 +264,15 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
             int c_idx = 0, fs = 0, fr = 0;      // convolution: channel block, filter column, filter row
             for (int kbi = 0; kbi < kl.num_kblocks;) {
-                if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                 const int nb = min(kl.nsub, kl.num_kblocks - kbi);
+                if (NPROD == 2 && (stage & 1) != pid) {
+                    // the other producer's slot: only keep the tap / channel counters in step
+                    for (int j = 0; j < nb; j++, kbi++)
+                        if (CONV && ++c_idx == kl.cblocks) { c_idx = 0; if (++fs == kl.S) { fs = 0; ++fr; } }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    continue;
+                }
+                if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                 const uint32_t full = bar_full + 8 * stage;
                 if (leader) mbar_expect_tx(full, nb * stage_tx);
                 for (int j = 0; j < nb; j++, kbi++) {
@@ -278,7 +293,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
         if (*s_stop) {
             // stopping early: let every copy this warp started land before the CTA retires
-            if (bres && blockIdx.x < sched.num_tiles && !mbar_wait_drain(bar_bres, 0, p.wait_limit_cycles))
+            if (bres && pid == 0 && blockIdx.x < sched.num_tiles && !mbar_wait_drain(bar_bres, 0, p.wait_limit_cycles))
                 atomicCAS(p.dev_status, 0u, (unsigned)DEV_TIMEOUT_DRAIN);
             for (int s = 0; s < STAGES; s++)
                 if (issued & (1u << s))
