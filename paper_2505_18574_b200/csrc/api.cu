@@ -204,8 +204,8 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
         }
     }
     switch (bn) {
-        case 256: return launch_tc<256, 4, false, 4, 1>(ctx, 0, tmA, tmB, p, st);
-        case 128: return launch_tc<128, 6, false, 4, 1>(ctx, 1, tmA, tmB, p, st);
+        case 256: return launch_tc<256, 4, false, 8, 1>(ctx, 0, tmA, tmB, p, st);
+        case 128: return launch_tc<128, 6, false, 8, 1>(ctx, 1, tmA, tmB, p, st);
         default:  return launch_tc<64, 8, false, 8, 1>(ctx, 2, tmA, tmB, p, st);
     }
 }
