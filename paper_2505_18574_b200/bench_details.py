@@ -17,11 +17,17 @@ import os
 import numpy as np
 
 ALL = ["0", "1a", "1b", "1c", "2", "3a", "3b", "3c", "4a", "4b"]
+# the shapes the paper prints: "g0".."g9" (inputs.SWEEP_GEMMS) and "c0", "c1" (inputs.SWEEP_CONVS)
+SWEEP = [f"g{i}" for i in range(10)] + ["c0", "c1"]
 L2_BYTES = 126e6
 
 
 def _problem(name):
     from . import inputs
+    if name[0] == "g":
+        return inputs.sweep_gemm(int(name[1:]))
+    if name[0] == "c":
+        return inputs.sweep_conv(int(name[1:]))
     return {"0": inputs.config0, "1a": lambda: inputs.config1(0), "1b": lambda: inputs.config1(1),
             "1c": lambda: inputs.config1(2), "2": inputs.config2, "3a": lambda: inputs.config3(0),
             "3b": lambda: inputs.config3(1), "3c": lambda: inputs.config3(2), "4a": inputs.config4a,
@@ -113,7 +119,7 @@ def run(dev=None, cfgs=None, iters=50, graph=True, peak_tops=None, peak_gbs=None
 
 if __name__ == "__main__":
     ap = argparse.ArgumentParser()
-    ap.add_argument("--cfg", default=",".join(ALL))
+    ap.add_argument("--cfg", default=",".join(ALL), help="comma list of configurations, or 'sweep' for the paper's printed shapes")
     ap.add_argument("--iters", type=int, default=50)
     ap.add_argument("--no-graph", action="store_true")
     a = ap.parse_args()
@@ -122,5 +128,6 @@ if __name__ == "__main__":
     peak_tops, peak_gbs = 2 * 1590.0, 6650.0
     if os.path.exists(pk):
         d = json.load(open(pk)); peak_tops, peak_gbs = 2 * d["bf16_tflops"], d["hbm_gbs"]
-    for r in run(cfgs=a.cfg.split(","), iters=a.iters, graph=not a.no_graph, peak_tops=peak_tops, peak_gbs=peak_gbs):
+    cfgs = SWEEP if a.cfg == "sweep" else a.cfg.split(",")
+    for r in run(cfgs=cfgs, iters=a.iters, graph=not a.no_graph, peak_tops=peak_tops, peak_gbs=peak_gbs):
         print(json.dumps(r), flush=True)

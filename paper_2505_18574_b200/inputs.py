@@ -201,3 +201,31 @@ def config4a() -> GemmProblem:
 def config4b() -> BatchedProblem:
     """16384 independent 64^3 GEMMs, tight row-major A/B/C, per-problem bias, shared mult/shift."""
     return make_batched(16384, 64, 64, 64, 104, name="cfg4b_batched_16384x64")
+
+
+# ---------------------------------------------------------------------------------------------
+# Shapes the paper itself prints (second workload): the Gemmini GEMM of its Code Examples
+# appendix, the schedule-reuse table (square / column-dominant / row-dominant GEMMs, read as
+# M x N x K with the listing's M=12544, K=256, N=64 for the column-dominant family), the
+# ablation's convolution (batch 4, 3x3, 14x14, 256 -> 256 channels) and, as int8 stand-ins, the
+# GEMM and conv2d shapes of its Trainium tables.  Seeds 200 + index; requantisation as config 1
+# for the GEMMs and as config 2 for the convolutions.
+# ---------------------------------------------------------------------------------------------
+SWEEP_GEMMS = [  # (M, N, K)
+    (12544, 64, 256), (1024, 1024, 1024), (512, 512, 512), (256, 256, 256), (6272, 64, 256), (12544, 64, 128),
+    (128, 1024, 1024), (64, 1024, 1024), (32, 1024, 1024), (4096, 8192, 8192),
+]
+SWEEP_CONVS = [  # (N, H, W, C, K, R, S, stride, pad)
+    (4, 14, 14, 256, 256, 3, 3, 1, 1),
+    (16, 128, 128, 128, 512, 3, 3, 1, 1),
+]
+
+
+def sweep_gemm(i: int) -> GemmProblem:
+    M, N, K = SWEEP_GEMMS[i]
+    return make_gemm(M, N, K, 200 + i, per_channel=1, relu=0, name=f"sweep_gemm_{M}x{N}x{K}")
+
+
+def sweep_conv(i: int) -> ConvProblem:
+    N, H, W, C, K, R, S, st, pad = SWEEP_CONVS[i]
+    return make_conv(N, H, W, C, K, R, S, st, pad, 300 + i, name=f"sweep_conv_{N}x{H}x{W}x{C}_k{K}_{R}x{S}")
