@@ -132,6 +132,26 @@ const char* i8_status_string(int status);
  * this library on the current device since the last call, or I8_ERR_CUDA.  Clears the record. */
 int i8ops_last_device_status(void* stream);
 
+/* Tile plan of gemm_i8's tensor path for one shape, and its reuse across shapes of the same aspect class: the
+ * analogue of the paper's schedule reuse (section "Improving Sample Efficiency With Schedule Reuse": a schedule found
+ * for one GEMM is replayed on GEMMs of the same aspect class: square, column-dominant, row-dominant). */
+typedef struct {
+    int shape_class;     /* 0 square (neither side 8x the other), 1 column-dominant (M >= 8N), 2 row-dominant (N >= 8M) */
+    int tile_m, tile_n;  /* output tile: 128 x {64, 128, 256} */
+    int stages;          /* ring slots of 128 bytes of K */
+    int m_tiles, n_tiles, waves;
+    int b_resident;      /* B fetched once per CTA and kept in shared memory */
+    int epilogue_warps;
+} i8_plan;
+
+/* Fills *out with the plan gemm_i8 would use for (M, N, K) on a device with sm_count SMs.  Host only; no CUDA call.
+ * Errors: I8_ERR_NULL, I8_ERR_SHAPE (a non-positive argument). */
+int i8ops_plan_gemm(int M, int N, int K, int sm_count, i8_plan* out);
+
+/* Records tile_n (64, 128 or 256; 0 forgets) as the tile width of every later shape of class shape_class, instead of
+ * the built-in cost model (a width wider than the problem is ignored).  Errors: I8_ERR_RANGE. */
+int i8ops_set_class_tile(int shape_class, int tile_n);
+
 /* Self-test of the failure path (no counterpart in the paper): launches one small CTA that waits, for at most
  * `limit_ms` (1..1000) milliseconds, on a barrier that nothing signals.  The kernel returns by itself and the next
  * i8ops_last_device_status() reports I8_ERR_TIMEOUT.  Nothing faults, traps or hangs. */

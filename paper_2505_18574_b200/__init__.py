@@ -5,9 +5,9 @@ every step of the computation runs in the CUDA kernels).  ``inputs`` holds the s
 ``build`` compiles the library with nvcc for sm_100a.
 """
 from .binding import (I8Error, batched_gemm_i8, conv2d_i8, gemm_i8, gemm_i8_host, last_device_status, last_path,
-                      lib, set_path, set_wait_limit_ms, status_string, PATH_GENERIC, PATH_NONE, PATH_SMALL,
+                      lib, plan_gemm, set_class_tile, set_path, set_wait_limit_ms, status_string, PATH_GENERIC, PATH_NONE, PATH_SMALL,
                       PATH_TENSOR)
 
 __all__ = ["I8Error", "batched_gemm_i8", "conv2d_i8", "gemm_i8", "gemm_i8_host", "last_device_status", "last_path",
-           "lib", "set_path", "set_wait_limit_ms", "status_string", "PATH_GENERIC", "PATH_NONE", "PATH_SMALL",
+           "lib", "plan_gemm", "set_class_tile", "set_path", "set_wait_limit_ms", "status_string", "PATH_GENERIC", "PATH_NONE", "PATH_SMALL",
            "PATH_TENSOR"]

@@ -30,6 +30,8 @@ SIGNATURES = {
     "i8_status_string": (ctypes.c_char_p, [_int]),
     "i8ops_last_device_status": (_int, [_vp]),
     "i8ops_selftest_bounded_wait": (_int, [_int, _vp]),
+    "i8ops_plan_gemm": (_int, [_int, _int, _int, _int, _vp]),
+    "i8ops_set_class_tile": (_int, [_int, _int]),
     "i8ops_last_cuda_error": (_int, []),
     "i8ops_last_path": (_int, []),
     "i8ops_set_path": (_int, [_int]),
@@ -130,6 +132,22 @@ def gemm_i8_host(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream
     st = lib().gemm_i8_host(hp(A), hp(B), hp(C), hp(bias), hp(mult), hp(shift), int(per_channel), M, N, K, int(relu),
                             _stream_ptr(stream))
     _check(st, "gemm_i8_host")
+
+
+class Plan(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("shape_class", "tile_m", "tile_n", "stages", "m_tiles", "n_tiles", "waves",
+                                             "b_resident", "epilogue_warps")]
+
+
+def plan_gemm(M: int, N: int, K: int, sm_count: int = 148) -> dict:
+    """The tile plan gemm_i8 would use for this shape (host-side query)."""
+    pl = Plan()
+    _check(lib().i8ops_plan_gemm(int(M), int(N), int(K), int(sm_count), ctypes.byref(pl)), "i8ops_plan_gemm")
+    return {n: getattr(pl, n) for n, _ in Plan._fields_}
+
+
+def set_class_tile(shape_class: int, tile_n: int) -> None:
+    _check(lib().i8ops_set_class_tile(int(shape_class), int(tile_n)), "i8ops_set_class_tile")
 
 
 def last_device_status(stream=None) -> int:

@@ -150,8 +150,20 @@ static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUt
 // Tile width.  Cost model in SM cycles: every wave of tiles pays, per 128-byte K block, an operand-delivery
 // bound of 256 + 2*BN, plus a fixed 400 per tile; the last tile's read-out (about 14 cycles per column) is
 // exposed.  The width with the lowest total wins; ties go to the wider tile.
+static int g_class_bn[3] = {0, 0, 0};            // per shape class: tile width recorded for reuse (0 = use the model)
+
+// Shape classes of the paper's schedule-reuse experiment: a schedule found for one shape is reused for shapes of the
+// same aspect class (square, column-dominant = tall and narrow, row-dominant = short and wide).
+static int shape_class(int M, int N) {
+    if ((int64_t)M >= 8 * (int64_t)N) return 1;
+    if ((int64_t)N >= 8 * (int64_t)M) return 2;
+    return 0;
+}
+
 static int choose_bn(int M, int N, int num_kb, int sm_count) {
     if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256) return g_force_bn;
+    const int recorded = g_class_bn[shape_class(M, N)];
+    if (recorded && (recorded == 64 || recorded - 64 < ((N + 63) / 64) * 64)) return recorded;
     const int cands[3] = {256, 128, 64};
     int best = 64;
     double best_cost = 1e300;
@@ -513,6 +525,31 @@ int i8ops_selftest_bounded_wait(int limit_ms, void* stream) {
     if (limit_ms > 1000) limit_ms = 1000;
     bounded_wait_selftest_kernel<<<1, 64, 0, (cudaStream_t)stream>>>((long long)limit_ms * 2000000ll, ctx->dev_status);
     CUDA_TRY(cudaGetLastError());
+    return I8_OK;
+}
+
+int i8ops_plan_gemm(int M, int N, int K, int sm_count, i8_plan* out) {
+    if (!out) return I8_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || sm_count <= 0) return I8_ERR_SHAPE;
+    const int num_kb = (K + BK - 1) / BK;
+    const int bn = choose_bn(M, N, num_kb, sm_count);
+    const int stages = bn == 256 ? 4 : (bn == 128 ? 6 : 8);
+    out->shape_class = shape_class(M, N);
+    out->tile_m = BM;
+    out->tile_n = bn;
+    out->stages = stages;
+    out->m_tiles = (M + BM - 1) / BM;
+    out->n_tiles = (N + bn - 1) / bn;
+    out->waves = (int)(((int64_t)out->m_tiles * out->n_tiles + sm_count - 1) / sm_count);
+    out->b_resident = (out->n_tiles == 1 && (int64_t)num_kb * bn * BK <= (int64_t)stages * bn * BK) ? 1 : 0;
+    out->epilogue_warps = 8;
+    return I8_OK;
+}
+
+int i8ops_set_class_tile(int shape_cls, int tile_n) {
+    if (shape_cls < 0 || shape_cls > 2) return I8_ERR_RANGE;
+    if (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) return I8_ERR_RANGE;
+    g_class_bn[shape_cls] = tile_n;
     return I8_OK;
 }
 

@@ -92,3 +92,35 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(binding, "_LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError):
         binding.lib()
+
+
+def test_tile_plan_and_class_reuse(L):
+    """Host-side plan query and the schedule-reuse analogue: shapes of one aspect class share a recorded tile."""
+    from paper_2505_18574_b200 import binding
+    # the paper's reuse table: base shape and its two reuse targets per class (M x N x K)
+    table = {0: [(1024, 1024, 1024), (512, 512, 512), (256, 256, 256)],
+             1: [(12544, 64, 256), (6272, 64, 256), (12544, 64, 128)],
+             2: [(128, 1024, 1024), (64, 1024, 1024), (32, 1024, 1024)]}
+    for cls, shapes in table.items():
+        for (M, N, K) in shapes:
+            pl = binding.plan_gemm(M, N, K)
+            assert pl["shape_class"] == cls and pl["tile_m"] == 128 and pl["tile_n"] in (64, 128, 256)
+            assert pl["m_tiles"] == -(-M // 128) and pl["n_tiles"] == -(-N // pl["tile_n"])
+            assert pl["waves"] == -(-(pl["m_tiles"] * pl["n_tiles"]) // 148)
+    assert binding.plan_gemm(12544, 64, 256)["b_resident"] == 1 and binding.plan_gemm(8192, 8192, 8192)["b_resident"] == 0
+    assert binding.plan_gemm(8192, 8192, 8192)["tile_n"] == 256
+    try:
+        base = binding.plan_gemm(1024, 1024, 1024)["tile_n"]
+        other = 128 if base != 128 else 64
+        binding.set_class_tile(0, other)                       # record a schedule for the square class ...
+        for (M, N, K) in table[0]:
+            assert binding.plan_gemm(M, N, K)["tile_n"] == other   # ... and every square shape reuses it
+        assert binding.plan_gemm(12544, 64, 256)["tile_n"] == 64   # other classes are untouched
+        binding.set_class_tile(1, 256)                         # wider than a 64-column problem: ignored
+        assert binding.plan_gemm(12544, 64, 256)["tile_n"] == 64
+    finally:
+        for c in range(3):
+            binding.set_class_tile(c, 0)
+    assert binding.plan_gemm(1024, 1024, 1024)["tile_n"] == base
+    assert L.i8ops_set_class_tile(3, 64) == 5 and L.i8ops_set_class_tile(0, 100) == 5
+    assert L.i8ops_plan_gemm(0, 1, 1, 148, None) == 1
