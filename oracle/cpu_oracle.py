@@ -49,6 +49,9 @@ def _bind(path: str):
                                          _int, _int, _int, _int, _int]
     L.oracle_conv2d_i8.restype = _int
     L.oracle_conv2d_i8.argtypes = [_i8p, _i8p, _i8p, _i32p, _i32p, _i32p, _int] + [_int] * 14
+    _dp = ctypes.POINTER(ctypes.c_double)
+    L.oracle_mpc_forward.restype = None
+    L.oracle_mpc_forward.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, _dp, _int, _int]
     L.oracle_num_threads.restype = _int
     L.oracle_num_threads.argtypes = []
     return L
@@ -119,6 +122,27 @@ class Oracle:
         return (y, int(ovf)) if return_overflow else y
 
 
+def _pd(a: Optional[np.ndarray]):
+    if a is None:
+        return ctypes.cast(None, ctypes.POINTER(ctypes.c_double))
+    assert a.dtype == np.float64 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _mpc_forward(self, Adyn, Bdyn, Kinf, x0, d, return_states: bool = False):
+    """u[batch, nhorizon, 4] (and x[batch, nhorizon, 12]) of the TinyMPC forward pass, evaluated in float64."""
+    f = lambda a: np.ascontiguousarray(a, dtype=np.float64)
+    Adyn, Bdyn, Kinf, x0, d = f(Adyn), f(Bdyn), f(Kinf), f(x0), f(d)
+    batch, nh = d.shape[0], d.shape[1]
+    assert Adyn.shape == (12, 12) and Bdyn.shape == (12, 4) and Kinf.shape == (4, 12) and x0.shape == (batch, 12) and d.shape[2] == 4
+    u = np.zeros((batch, nh, 4), dtype=np.float64)
+    xs = np.zeros((batch, nh, 12), dtype=np.float64) if return_states else None
+    self._L.oracle_mpc_forward(_pd(Adyn), _pd(Bdyn), _pd(Kinf), _pd(x0), _pd(d), _pd(u), _pd(xs), batch, nh)
+    return (u, xs) if return_states else u
+
+
+Oracle.mpc_forward = _mpc_forward
+
 _default: Optional[Oracle] = None
 
 
@@ -152,3 +176,7 @@ def batched_gemm_i8(*a, **k):
 
 def conv2d_i8(*a, **k):
     return lib().conv2d_i8(*a, **k)
+
+
+def mpc_forward(*a, **k):
+    return lib().mpc_forward(*a, **k)

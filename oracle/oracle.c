@@ -187,3 +187,44 @@ int oracle_num_threads(void)
     return 1;
 #endif
 }
+
+/* ------------------------------------------------------------------------------------------------------
+ * Fine-grained linear algebra: the forward pass of the TinyMPC primal update that the paper optimises
+ * (Code Examples appendix, "TinyMPC Primal Update Forward Pass"; Evaluation, "Fine-Grained Linear Algebra"):
+ *     u[i]   = -Kinf * x[i] - d[i]
+ *     x[i+1] =  Adyn * x[i] + Bdyn * u[i]            i = 0 .. nhorizon-1
+ * Adyn is 12x12, Bdyn 12x4, Kinf 4x12 (row-major), x[0] and d are inputs, u is the output; the last state
+ * x[nhorizon] is not needed and not formed.  The paper runs it in fp32 on one instance; here `batch`
+ * independent instances share the three matrices.  The oracle evaluates the two equations in double
+ * precision, in the plain order written above.  xs (optional, may be NULL) receives x[0..nhorizon-1].
+ */
+#define MPC_NX 12
+#define MPC_NU 4
+void oracle_mpc_forward(const double *Adyn, const double *Bdyn, const double *Kinf,
+                        const double *x0, const double *d, double *u, double *xs, int batch, int nhorizon)
+{
+    #pragma omp parallel for schedule(static)
+    for (int b = 0; b < batch; b++) {
+        double x[MPC_NX], xn[MPC_NX];
+        for (int r = 0; r < MPC_NX; r++) x[r] = x0[(int64_t)b * MPC_NX + r];
+        for (int i = 0; i < nhorizon; i++) {
+            double *ui = u + ((int64_t)b * nhorizon + i) * MPC_NU;
+            const double *di = d + ((int64_t)b * nhorizon + i) * MPC_NU;
+            if (xs) for (int r = 0; r < MPC_NX; r++) xs[((int64_t)b * nhorizon + i) * MPC_NX + r] = x[r];
+            for (int r = 0; r < MPC_NU; r++) {
+                double kx = 0.0;
+                for (int c = 0; c < MPC_NX; c++) kx += Kinf[r * MPC_NX + c] * x[c];
+                ui[r] = -kx - di[r];
+            }
+            if (i + 1 < nhorizon) {
+                for (int r = 0; r < MPC_NX; r++) {
+                    double ax = 0.0, bu = 0.0;
+                    for (int c = 0; c < MPC_NX; c++) ax += Adyn[r * MPC_NX + c] * x[c];
+                    for (int c = 0; c < MPC_NU; c++) bu += Bdyn[r * MPC_NU + c] * ui[c];
+                    xn[r] = ax + bu;
+                }
+                for (int r = 0; r < MPC_NX; r++) x[r] = xn[r];
+            }
+        }
+    }
+}

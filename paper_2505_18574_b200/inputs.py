@@ -229,3 +229,33 @@ def sweep_gemm(i: int) -> GemmProblem:
 def sweep_conv(i: int) -> ConvProblem:
     N, H, W, C, K, R, S, st, pad = SWEEP_CONVS[i]
     return make_conv(N, H, W, C, K, R, S, st, pad, 300 + i, name=f"sweep_conv_{N}x{H}x{W}x{C}_k{K}_{R}x{S}")
+
+
+# ---------------------------------------------------------------------------------------------
+# Fine-grained linear algebra as the paper runs it: the TinyMPC primal-update forward pass
+# (12 states, 4 inputs, NHORIZON = 5, fp32).  The paper's controller matrices are not available;
+# the stand-ins are a stable random system: Adyn = I + 0.05*G (G standard normal), Bdyn = 0.1*G,
+# Kinf = 0.3*G, initial states and d uniform on [-1, 1].  `batch` independent instances share
+# the three matrices.
+# ---------------------------------------------------------------------------------------------
+@dataclass
+class MpcProblem:
+    name: str
+    batch: int
+    nhorizon: int
+    Adyn: np.ndarray   # float32 [12, 12]
+    Bdyn: np.ndarray   # float32 [12, 4]
+    Kinf: np.ndarray   # float32 [4, 12]
+    x0: np.ndarray     # float32 [batch, 12]
+    d: np.ndarray      # float32 [batch, nhorizon, 4]
+    seed: int = 0
+
+
+def make_mpc(batch: int, nhorizon: int = 5, seed: int = 5, name=None) -> MpcProblem:
+    rng = np.random.Generator(np.random.PCG64(seed))
+    Adyn = (np.eye(12) + 0.05 * rng.standard_normal((12, 12))).astype(np.float32)
+    Bdyn = (0.1 * rng.standard_normal((12, 4))).astype(np.float32)
+    Kinf = (0.3 * rng.standard_normal((4, 12))).astype(np.float32)
+    x0 = rng.uniform(-1.0, 1.0, size=(batch, 12)).astype(np.float32)
+    d = rng.uniform(-1.0, 1.0, size=(batch, nhorizon, 4)).astype(np.float32)
+    return MpcProblem(name or f"mpc_forward_{batch}x{nhorizon}", batch, nhorizon, Adyn, Bdyn, Kinf, x0, d, seed)
