@@ -132,6 +132,20 @@ const char* i8_status_string(int status);
  * this library on the current device since the last call, or I8_ERR_CUDA.  Clears the record. */
 int i8ops_last_device_status(void* stream);
 
+/*
+ * Forward pass of the TinyMPC primal update, the paper's fine-grained linear-algebra benchmark (Code Examples
+ * appendix, "TinyMPC Primal Update Forward Pass"), for `batch` independent instances that share the matrices:
+ *     u[i] = -Kinf * x[i] - d[i];   x[i+1] = Adyn * x[i] + Bdyn * u[i];   i = 0 .. nhorizon-1  (x[nhorizon] is not formed)
+ *   Adyn [12][12], Bdyn [12][4], Kinf [4][12]   HOST pointers, row-major fp32 (copied into the launch's arguments)
+ *   x0 [batch][12], d [batch][nhorizon][4]      device, fp32, 16-byte aligned
+ *   u  [batch][nhorizon][4]                     device output, fp32, 16-byte aligned
+ *   xs [batch][nhorizon][12] or NULL            device output: the states x[0..nhorizon-1]
+ * Arithmetic is fp32 with fused multiply-adds in ascending index order (the paper's precision).
+ * Errors: I8_ERR_SHAPE (negative batch or nhorizon), I8_ERR_NULL, I8_ERR_ALIGN, I8_ERR_CUDA.
+ */
+int mpc_forward_f32(const float* Adyn, const float* Bdyn, const float* Kinf, const float* x0, const float* d, float* u,
+                    float* xs, int batch, int nhorizon, void* stream);
+
 /* Tile plan of gemm_i8's tensor path for one shape, and its reuse across shapes of the same aspect class: the
  * analogue of the paper's schedule reuse (section "Improving Sample Efficiency With Schedule Reuse": a schedule found
  * for one GEMM is replayed on GEMMs of the same aspect class: square, column-dominant, row-dominant). */

@@ -1,5 +1,6 @@
 """Per-problem timings of every workload configuration (GEMM 256^3, the three large GEMMs, the four
-convolutions, the tall-skinny GEMM and the batched 64^3 products) through the C-ABI binding.
+convolutions, the tall-skinny GEMM and the batched 64^3 products; `--cfg mpc` adds the fp32 TinyMPC forward pass over
+2^20 instances and `--cfg sweep` the shapes the paper prints) through the C-ABI binding.
 
     python -m paper_2505_18574_b200.bench_details [--cfg 0,1a,2,...] [--iters N] [--no-graph]
 
@@ -16,7 +17,7 @@ import os
 
 import numpy as np
 
-ALL = ["0", "1a", "1b", "1c", "2", "3a", "3b", "3c", "4a", "4b"]
+ALL = ["0", "1a", "1b", "1c", "2", "3a", "3b", "3c", "4a", "4b", "mpc"]
 # the shapes the paper prints: "g0".."g9" (inputs.SWEEP_GEMMS) and "c0", "c1" (inputs.SWEEP_CONVS)
 SWEEP = [f"g{i}" for i in range(10)] + ["c0", "c1"]
 L2_BYTES = 126e6
@@ -24,6 +25,8 @@ L2_BYTES = 126e6
 
 def _problem(name):
     from . import inputs
+    if name == "mpc":
+        return inputs.make_mpc(1 << 20)
     if name[0] == "g":
         return inputs.sweep_gemm(int(name[1:]))
     if name[0] == "c":
@@ -64,6 +67,16 @@ def _make(name, dev, copies_for_l2=True):
         def launch(i):
             x, w, y = bufs[i % sets]
             i8.conv2d_i8(x, w, y, b, mu, sh, p.per_channel, p.relu, (p.stride_h, p.stride_w), (p.pad_h, p.pad_w))
+    elif isinstance(p, inputs.MpcProblem):
+        # flops: per step 2*4*12 + 4 (u) and 2*12*12 + 2*12*4 + 12 (x), the last step without the state update
+        ops = p.batch * (p.nhorizon * 100.0 + (p.nhorizon - 1) * 396.0)
+        byts = p.batch * (48 + 32 * p.nhorizon)
+        sets = 1
+        x0, d = T(p.x0), T(p.d)
+        u = torch.empty((p.batch, p.nhorizon, 4), dtype=torch.float32, device=dev)
+
+        def launch(i):
+            i8.mpc_forward_f32(p.Adyn, p.Bdyn, p.Kinf, x0, d, u)
     else:
         ops = 2.0 * p.batch * p.M * p.N * p.K
         byts = p.A.size + p.B.size + p.batch * p.M * p.N + p.bias.size * 4

@@ -27,6 +27,7 @@ SIGNATURES = {
                                _int, _int, _int, _int, _int, _vp]),
     "conv2d_i8": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int] + [_int] * 12 + [_vp]),
     "gemm_i8_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
+    "mpc_forward_f32": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp]),
     "i8_status_string": (ctypes.c_char_p, [_int]),
     "i8ops_last_device_status": (_int, [_vp]),
     "i8ops_selftest_bounded_wait": (_int, [_int, _vp]),
@@ -132,6 +133,19 @@ def gemm_i8_host(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream
     st = lib().gemm_i8_host(hp(A), hp(B), hp(C), hp(bias), hp(mult), hp(shift), int(per_channel), M, N, K, int(relu),
                             _stream_ptr(stream))
     _check(st, "gemm_i8_host")
+
+
+def mpc_forward_f32(Adyn, Bdyn, Kinf, x0, d, u, xs=None, stream=None) -> None:
+    """TinyMPC forward pass.  Adyn (12,12), Bdyn (12,4), Kinf (4,12): host float32 arrays (numpy or CPU tensors);
+    x0 (batch,12), d (batch,nh,4), u (batch,nh,4) and optional xs (batch,nh,12): contiguous CUDA float32 tensors."""
+    import numpy as np
+    mats = [np.ascontiguousarray(np.asarray(a), dtype=np.float32) for a in (Adyn, Bdyn, Kinf)]
+    assert mats[0].shape == (12, 12) and mats[1].shape == (12, 4) and mats[2].shape == (4, 12)
+    batch, nh = d.shape[0], d.shape[1]
+    assert tuple(x0.shape) == (batch, 12) and tuple(u.shape) == (batch, nh, 4) and x0.is_contiguous() and d.is_contiguous()
+    st = lib().mpc_forward_f32(mats[0].ctypes.data, mats[1].ctypes.data, mats[2].ctypes.data, _ptr(x0), _ptr(d), _ptr(u),
+                               _ptr(xs), batch, nh, _stream_ptr(stream))
+    _check(st, "mpc_forward_f32")
 
 
 class Plan(ctypes.Structure):

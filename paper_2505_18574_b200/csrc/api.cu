@@ -13,6 +13,7 @@
 #include "batched_tc.cuh"
 #include "gemm_tc.cuh"
 #include "generic.cuh"
+#include "mpc.cuh"
 
 namespace i8 {
 
@@ -525,6 +526,29 @@ int i8ops_selftest_bounded_wait(int limit_ms, void* stream) {
     if (limit_ms > 1000) limit_ms = 1000;
     bounded_wait_selftest_kernel<<<1, 64, 0, (cudaStream_t)stream>>>((long long)limit_ms * 2000000ll, ctx->dev_status);
     CUDA_TRY(cudaGetLastError());
+    return I8_OK;
+}
+
+int mpc_forward_f32(const float* Adyn, const float* Bdyn, const float* Kinf, const float* x0, const float* d, float* u,
+                    float* xs, int batch, int nhorizon, void* stream) {
+    t_last_path = I8_PATH_NONE;
+    if (batch < 0 || nhorizon < 0) return I8_ERR_SHAPE;
+    if (batch == 0 || nhorizon == 0) return I8_OK;
+    if (!Adyn || !Bdyn || !Kinf || !x0 || !d || !u) return I8_ERR_NULL;
+    if (!aligned16(x0) || !aligned16(d) || !aligned16(u) || (xs && !aligned16(xs))) return I8_ERR_ALIGN;
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    MpcMatrices m;
+    memcpy(m.A, Adyn, sizeof(m.A));
+    memcpy(m.B, Bdyn, sizeof(m.B));
+    memcpy(m.K, Kinf, sizeof(m.K));
+    int blocks = (batch + 127) / 128;
+    if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
+    cudaStream_t st = (cudaStream_t)stream;
+    mpc_forward_f32_kernel<<<blocks, 128, 0, st>>>(m, (const float4*)x0, (const float4*)d, (float4*)u, (float4*)xs, batch, nhorizon);
+    CUDA_TRY(cudaGetLastError());
+    t_last_path = I8_PATH_GENERIC;
     return I8_OK;
 }
 
