@@ -85,6 +85,19 @@ int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs,
             int M, int N, int K, int relu, void* stream);
 
 /*
+ * Raw read-out: D[m*ldd + n] (+)= sum_k A[..] * B[..] as int32, with no bias, activation or scale.  This is the
+ * accumulator read as accumulator-type data (Gemmini ISA description, continued: address bit 29 set), and with
+ * accumulate != 0 the product is added to what D already holds (address bit 30: accumulate instead of overwrite),
+ * which lets a caller split K across calls.  D is device int32, row-major, ldd >= N; other arguments as gemm_i8.
+ * The sums must fit in int32 (always true for a single product with K <= 65536).
+ * Errors: I8_ERR_NULL, I8_ERR_SHAPE, I8_ERR_STRIDE, I8_ERR_RANGE, I8_ERR_CUDA.
+ */
+int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs,
+                const int8_t* B, int64_t b_rs, int64_t b_cs,
+                int32_t* D, int64_t ldd, int accumulate,
+                int M, int N, int K, void* stream);
+
+/*
  * `batch` independent products (the paper's fine-grained linear algebra: many small, low-reuse
  * products, Evaluation "Fine-Grained Linear Algebra"; also its column-dominant GEMM shapes).
  * Problem b uses A + b*a_bs, B + b*b_bs, C + b*c_bs and bias + b*bias_bs (bias_bs == 0: one bias

@@ -23,6 +23,7 @@ _int = ctypes.c_int
 # name -> (restype, argtypes); every symbol that include/i8ops.h declares
 SIGNATURES = {
     "gemm_i8": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
+    "gemm_i8_raw": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _int, _int, _int, _int, _vp]),
     "batched_gemm_i8": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _int,
                                _int, _int, _int, _int, _int, _vp]),
     "conv2d_i8": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int] + [_int] * 12 + [_vp]),
@@ -94,6 +95,16 @@ def gemm_i8(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None
     st = lib().gemm_i8(_ptr(A), A.stride(0), A.stride(1), _ptr(B), B.stride(0), B.stride(1), _ptr(C), C.stride(0),
                        _ptr(bias), _ptr(mult), _ptr(shift), int(per_channel), M, N, K, int(relu), _stream_ptr(stream))
     _check(st, "gemm_i8")
+
+
+def gemm_i8_raw(A, B, D, accumulate: bool = False, stream=None) -> None:
+    """D (+)= A . B as int32 accumulators (no epilogue).  A: (M, K), B: (K, N) int8 views, D: (M, N) int32."""
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2 and tuple(D.shape) == (M, N) and (D.stride(1) == 1 or N <= 1)
+    st = lib().gemm_i8_raw(_ptr(A), A.stride(0), A.stride(1), _ptr(B), B.stride(0), B.stride(1), _ptr(D), D.stride(0),
+                           int(bool(accumulate)), M, N, K, _stream_ptr(stream))
+    _check(st, "gemm_i8_raw")
 
 
 def batched_gemm_i8(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:

@@ -182,9 +182,11 @@ static int choose_bn(int M, int N, int num_kb, int sm_count) {
 
 // Common tail of the tensor paths: B's tensor map (an N x K matrix with K contiguous), the tile schedule,
 // and the launch of the instance that matches the tile width.
+struct RawOut { int32_t* D = nullptr; int64_t ldd = 0; int accumulate = 0; };
+
 static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop& kl, int bn, const int8_t* B, int64_t ldb,
                   int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
-                  int M, int N, int K, int relu, cudaStream_t st) {
+                  int M, int N, int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
     CUtensorMap tmB;
     {
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
@@ -196,7 +198,8 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
     GemmTcParams p;
     p.C = C; p.ldc = ldc; p.bias = bias; p.mult = mult; p.shift = shift;
     p.per_channel = per_channel; p.relu = relu; p.M = M; p.N = N; p.K = K;
-    p.c_vec_ok = aligned16(C) && (ldc % 16 == 0);
+    p.c_vec_ok = raw.D ? (aligned16(raw.D) && raw.ldd % 4 == 0) : (aligned16(C) && (ldc % 16 == 0));
+    p.D = raw.D; p.ldd = raw.ldd; p.raw = raw.D ? 1 : 0; p.accumulate = raw.accumulate;
     p.sched.m_tiles = (M + BM - 1) / BM;
     p.sched.n_tiles = (N + bn - 1) / bn;
     p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
@@ -225,7 +228,7 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
 
 static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
-                       int K, int relu, cudaStream_t st) {
+                       int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
     const int bn = choose_bn(M, N, (K + BK - 1) / BK, ctx->sm_count);
     CUtensorMap tmA;
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
@@ -237,7 +240,7 @@ static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_
     kl.cb = BK; kl.nsub = 1; kl.num_kblocks = (K + BK - 1) / BK;
     kl.num_iters = kl.num_kblocks;
     kl.mmas_last = ((K - (kl.num_iters - 1) * BK) + 31) / 32;
-    return run_tc(ctx, false, tmA, kl, bn, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
+    return run_tc(ctx, false, tmA, kl, bn, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
 }
 
 // Implicit-GEMM convolution: A tiles come from an im2col-mode tensor map over the NHWC activations.
@@ -362,7 +365,34 @@ int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_
         if (rc == I8_OK) t_last_path = I8_PATH_TENSOR;
         return rc;
     }
-    GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, C, ldc, 0, bias, 0, mult, shift, per_channel, relu, 1, M, N, K};
+    GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, C, ldc, 0, bias, 0, mult, shift, per_channel, relu, 1, M, N, K, nullptr, 0, 0, 0};
+    rc = run_gemm_generic(g, st);
+    if (rc == I8_OK) t_last_path = I8_PATH_GENERIC;
+    return rc;
+}
+
+int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_t b_rs, int64_t b_cs, int32_t* D, int64_t ldd,
+                int accumulate, int M, int N, int K, void* stream) {
+    t_last_path = I8_PATH_NONE;
+    if (M < 0 || N < 0 || K < 0) return I8_ERR_SHAPE;
+    if (K > 65536) return I8_ERR_RANGE;
+    if (M == 0 || N == 0) return I8_OK;
+    if (!D || (K > 0 && (!A || !B))) return I8_ERR_NULL;
+    if (!strides_ok(a_rs, a_cs, M, K) || !strides_ok(b_rs, b_cs, K, N) || ldd < N) return I8_ERR_STRIDE;
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool tc_legal = K >= 1 && a_cs == 1 && b_rs == 1 && aligned16(A) && aligned16(B) && a_rs % 16 == 0 &&
+                          b_cs % 16 == 0 && a_rs >= K && b_cs >= K;
+    if (tc_legal && g_path_mode != 1) {
+        RawOut raw; raw.D = D; raw.ldd = ldd; raw.accumulate = accumulate ? 1 : 0;
+        rc = run_gemm_tc(ctx, A, a_rs, B, b_cs, nullptr, 0, nullptr, nullptr, nullptr, 0, M, N, K, 0, st, raw);
+        if (rc == I8_OK) t_last_path = I8_PATH_TENSOR;
+        return rc;
+    }
+    GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, nullptr, 0, 0, nullptr, 0, nullptr, nullptr, 0, 0, 1, M, N, K,
+                        D, ldd, 1, accumulate ? 1 : 0};
     rc = run_gemm_generic(g, st);
     if (rc == I8_OK) t_last_path = I8_PATH_GENERIC;
     return rc;
@@ -394,7 +424,7 @@ int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs, c
         }
     }
     GenericGemmParams g{A, a_rs, a_cs, a_bs, B, b_rs, b_cs, b_bs, C, ldc, c_bs, bias, bias_bs, mult, shift, per_channel, relu,
-                        batch, M, N, K};
+                        batch, M, N, K, nullptr, 0, 0, 0};
     rc = run_gemm_generic(g, st);
     if (rc == I8_OK) t_last_path = I8_PATH_GENERIC;
     return rc;

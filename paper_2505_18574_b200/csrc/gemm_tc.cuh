@@ -67,7 +67,10 @@ struct GemmTcParams {
     const int32_t* shift;
     int per_channel, relu;
     int M, N, K;
-    int c_vec_ok;               // C and ldc are 16-byte aligned: full chunks go out as 16-byte stores
+    int c_vec_ok;               // C (or D) and its leading dimension are 16-byte aligned: full chunks go out as 16-byte stores
+    int32_t* D;                 // raw read-out: the int32 accumulators themselves, no bias / activation / scale
+    int64_t ldd;
+    int raw, accumulate;        // raw != 0 selects D; accumulate != 0 adds to what D already holds
     TileSched sched;
     KLoop kl;
     long long wait_limit_cycles;
@@ -144,6 +147,23 @@ __device__ __forceinline__ void store_row_chunk(int8_t* crow, int n, int N, bool
 #pragma unroll
         for (int j = 0; j < 32; j++)
             if (n + j < N) crow[n + j] = (int8_t)((out[j >> 2] >> (8 * (j & 3))) & 0xff);
+    }
+}
+
+// Raw read-out of one thread's 32 accumulators (columns n .. n+31 of one row), optionally added to the destination.
+__device__ __forceinline__ void store_raw_chunk(int32_t* drow, int n, int N, bool vec_ok, bool accumulate, const int32_t (&v)[32]) {
+    if (vec_ok && n + 32 <= N) {
+        int4* dst = reinterpret_cast<int4*>(drow + n);
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            int4 o = make_int4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            if (accumulate) { const int4 e = dst[j]; o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+            dst[j] = o;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; j++)
+            if (n + j < N) drow[n + j] = accumulate ? drow[n + j] + v[j] : v[j];
     }
 }
 
@@ -382,7 +402,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 for (int c = etid; c < BN; c += EPI_THREADS) {
                     const int n = n0 + c;
                     int32_t bias = 0, mult = 0, shift = 0;
-                    if (n < p.N) {
+                    if (n < p.N && !p.raw) {
                         bias = p.bias ? p.bias[n] : 0;
                         mult = p.mult[p.per_channel ? n : 0];
                         shift = p.shift[p.per_channel ? n : 0];
@@ -418,6 +438,12 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 int32_t v[32];
                 tmem_ld_32x32(t0 + c0, v);
                 tmem_ld_wait();
+                if (p.raw) {
+                    // the accumulator read as accumulator-type data (Gemmini's unscaled read-out), optionally
+                    // accumulated on top of the destination (its accumulate-on-write mode)
+                    if (row < p.M) store_raw_chunk(p.D + (int64_t)row * p.ldd, n, p.N, p.c_vec_ok != 0, p.accumulate != 0, v);
+                    continue;
+                }
                 uint32_t out[8];
                 if (shift32) {
                     if constexpr (ONE_CHUNK) {

@@ -15,6 +15,7 @@ struct GenericGemmParams {
     const int32_t* mult; const int32_t* shift;
     int per_channel, relu;
     int batch, M, N, K;
+    int32_t* D; int64_t ldd; int raw, accumulate;   // raw read-out of the accumulators (see gemm_i8_raw)
 };
 
 __global__ void __launch_bounds__(256) gemm_i8_generic_kernel(const GenericGemmParams p) {
@@ -28,6 +29,11 @@ __global__ void __launch_bounds__(256) gemm_i8_generic_kernel(const GenericGemmP
         const int8_t* bb = p.B + b * p.b_bs + (int64_t)n * p.b_cs;
         int32_t acc = 0;
         for (int k = 0; k < p.K; k++) acc += (int32_t)a[(int64_t)k * p.a_cs] * (int32_t)bb[(int64_t)k * p.b_rs];
+        if (p.raw) {
+            int32_t* dst = p.D + (int64_t)m * p.ldd + n;
+            *dst = p.accumulate ? *dst + acc : acc;
+            continue;
+        }
         const int32_t bias = p.bias ? p.bias[b * p.bias_bs + n] : 0;
         const int ci = p.per_channel ? n : 0;
         p.C[b * p.c_bs + (int64_t)m * p.ldc + n] = (int8_t)requant_wide(acc, bias, p.relu, p.mult[ci], p.shift[ci]);

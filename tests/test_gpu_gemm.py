@@ -151,3 +151,31 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     assert i8.last_device_status() == 0            # the record is cleared by the query
     p = inputs.make_gemm(128, 64, 64, 3, per_channel=0, relu=1)
     H.assert_same(H.gemm_gpu(p), H.gemm_oracle(p), "gemm after a timed-out wait")
+
+
+@pytest.mark.parametrize("M,N,K,ldd_pad", [(128, 256, 128, 0), (300, 200, 112, 4), (513, 96, 1040, 0), (64, 40, 48, 3), (1000, 1024, 512, 0)])
+def test_raw_accumulator_readout_and_split_k(M, N, K, ldd_pad):
+    """gemm_i8_raw returns the int32 sums themselves; two accumulate calls over halves of K equal one call over all of K."""
+    import torch
+    import oracle
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_gemm(M, N, K, 70 + M, per_channel=0, relu=0)
+    want = oracle.gemm_acc(p.A, p.a_rs, 1, p.B, 1, p.b_cs, M, N, K).astype(np.int32)
+    A = torch.from_numpy(p.A).cuda(); B = torch.from_numpy(p.B).cuda()
+    for mode in (0, 1):
+        i8.set_path(mode)
+        Dbuf = torch.full((M, N + ldd_pad), 77, dtype=torch.int32, device="cuda")
+        D = Dbuf[:, :N]
+        i8.gemm_i8_raw(A, B.t(), D)
+        assert i8.last_device_status() == 0
+        assert i8.last_path() == (i8.PATH_TENSOR if mode == 0 else i8.PATH_GENERIC)
+        H.assert_same(D.cpu().numpy(), want, f"raw mode {mode}")
+        if ldd_pad:
+            assert (Dbuf[:, N:] == 77).all()
+        kh = (K // 32) * 16                     # split K at a multiple of 16 so both halves stay on the tensor path
+        if kh:
+            D.zero_()
+            i8.gemm_i8_raw(A[:, :kh], B[:, :kh].t(), D, accumulate=True)
+            i8.gemm_i8_raw(A[:, kh:], B[:, kh:].t(), D, accumulate=True)
+            H.assert_same(D.cpu().numpy(), want, f"split-K accumulate mode {mode}")
+    i8.set_path(0)
