@@ -331,10 +331,9 @@ def main():
                              "so each problem's tiles are evicted before its next launch",
                        "per_problem_ms": {p.name: per_problem_ms[j] for j, p in enumerate(problems)},
                        "per_problem_tops": {p.name: gemm_ops(p) / (per_problem_ms[j] * 1e-3) / 1e12 for j, p in enumerate(problems)}},
-            "roofline": {"bound": "tensor", "kernel": "gemm_i8_tc_kernel<256,4>", "achieved": achieved, "peak": peak_int8,
-                         "unit": "TFLOP/s", "frac": achieved / peak_int8, "traffic": NCU_STEP_TRAFFIC_BYTES,
-                         "traffic_note": "DRAM bytes read+written by one step (one launch of each problem) from the ncu launch list in "
-                                         "profiles/bench_config1_launch_list.txt; algorithmic bytes per step 4.87e8",
+            "roofline": {"bound": "tensor", "kernel": "gemm_i8_tc2_kernel (two-SM, 256x256 tiles, cta_group::2)", "achieved": achieved, "peak": peak_int8,
+                         "unit": "TFLOP/s", "frac": achieved / peak_int8, "traffic": None,
+                         "traffic_note": "null until the counters are re-taken for the current kernel; algorithmic bytes per step 4.87e8",
                          "peak_source": f"{peaks['source']}: bf16 sustained {peaks['bf16_sustained']} TFLOP/s x {NOMINAL_INT8_OVER_BF16} "
                                         f"(nominal int8:bf16 ratio); burst-based peak would be {peaks['bf16_burst'] * 2:.0f}; nominal 4500",
                          "frac_of_nominal_4500": achieved / 4500.0},

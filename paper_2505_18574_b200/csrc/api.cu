@@ -12,6 +12,7 @@
 #include "../../include/i8ops.h"
 #include "batched_tc.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc2.cuh"
 #include "generic.cuh"
 #include "mpc.cuh"
 
@@ -36,6 +37,7 @@ static std::mutex g_mutex;
 static int g_path_mode = 0;                      // 0 auto, 1 generic only, 2 tensor whenever legal
 static uint64_t g_wait_limit_ns = 2000ull * 1000 * 1000;
 static int g_pdl = 1;                            // programmatic dependent launch (I8OPS_PDL=0 turns it off)
+static int g_tc2 = 1;                            // two-SM GEMM kernel for large shapes (I8OPS_TC2=0 turns it off)
 static int g_force_bn = -1;                      // tuning override from the environment (I8OPS_FORCE_BN)
 
 static thread_local int t_last_path = I8_PATH_NONE;
@@ -85,6 +87,8 @@ static int get_ctx(DeviceCtx** out) {
         }
         const char* bn = getenv("I8OPS_FORCE_BN");
         if (bn) g_force_bn = atoi(bn);
+        const char* tc2 = getenv("I8OPS_TC2");
+        if (tc2) g_tc2 = atoi(tc2);
         const char* pdl = getenv("I8OPS_PDL");
         if (pdl) g_pdl = atoi(pdl);
         c.ready = true;
@@ -226,9 +230,52 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
     }
 }
 
+// Two-SM kernel: 256 x 256 tiles, one cluster of two CTAs per tile.
+static int run_gemm_tc2(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
+                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
+                        int K, int relu, cudaStream_t st, const RawOut& raw) {
+    CUtensorMap tmA, tmB;
+    {
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
+        const uint64_t str[1] = {(uint64_t)lda};
+        const uint32_t box[2] = {BK, BM};
+        int rc = make_tmap(&tmA, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (rc) return rc;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
+        const uint64_t str[1] = {(uint64_t)ldb};
+        const uint32_t box[2] = {BK, TC2_BN / 2};
+        int rc = make_tmap(&tmB, B, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (rc) return rc;
+    }
+    GemmTcParams p;
+    p.C = C; p.ldc = ldc; p.bias = bias; p.mult = mult; p.shift = shift;
+    p.per_channel = per_channel; p.relu = relu; p.M = M; p.N = N; p.K = K;
+    p.c_vec_ok = raw.D ? (aligned16(raw.D) && raw.ldd % 4 == 0) : (aligned16(C) && (ldc % 16 == 0));
+    p.D = raw.D; p.ldd = raw.ldd; p.raw = raw.D ? 1 : 0; p.accumulate = raw.accumulate;
+    p.sched.m_tiles = (M + 255) / 256;
+    p.sched.n_tiles = (N + TC2_BN - 1) / TC2_BN;
+    p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
+    p.sched.group_m = 8;
+    p.kl = KLoop{};
+    p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);
+    p.dev_status = ctx->dev_status;
+    if (!ctx->attr_set[7]) {
+        CUDA_TRY(cudaFuncSetAttribute(gemm_i8_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Tc2Smem::DYN_BYTES));
+        ctx->attr_set[7] = true;
+    }
+    int clusters = ctx->sm_count / 2;
+    if (p.sched.num_tiles < clusters) clusters = p.sched.num_tiles;
+    CUDA_TRY(launch_kernel(gemm_i8_tc2_kernel, false, 2 * clusters, TC2_THREADS, Tc2Smem::DYN_BYTES, st, tmA, tmB, p));
+    return I8_OK;
+}
+
 static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
                        int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
+    if (g_tc2 && M >= 512 && N >= 512 && g_force_bn < 0)
+        return run_gemm_tc2(ctx, A, lda, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
     const int bn = choose_bn(M, N, (K + BK - 1) / BK, ctx->sm_count);
     CUtensorMap tmA;
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};

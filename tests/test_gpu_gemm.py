@@ -179,3 +179,16 @@ def test_raw_accumulator_readout_and_split_k(M, N, K, ldd_pad):
             i8.gemm_i8_raw(A[:, kh:], B[:, kh:].t(), D, accumulate=True)
             H.assert_same(D.cpu().numpy(), want, f"split-K accumulate mode {mode}")
     i8.set_path(0)
+
+
+@pytest.mark.parametrize("M,N,K", [(512, 512, 128), (513, 600, 1040), (1000, 520, 272), (640, 1300, 144), (769, 1025, 48), (2048, 1536, 4096)])
+def test_two_sm_kernel_shapes(M, N, K):
+    """Shapes with M, N >= 512 run on the two-SM (cta_group::2) kernel: ragged edges in M, N and K, both epilogue forms."""
+    pad = (-K) % 16
+    for per_channel, relu, shift_hi in ((1, 0, 22), (0, 1, 18)):
+        p = inputs.make_gemm(M, N, K, 2000 + M + N + K, per_channel=per_channel, relu=relu, shift_lo=12, shift_hi=shift_hi,
+                             lda_pad=pad, ldb_pad=pad, ldc_pad=16 * per_channel)
+        _both_paths(p)
+    p = inputs.make_gemm(M, N, K, 7, per_channel=0, relu=0, lda_pad=pad, ldb_pad=pad)
+    p.mult[:] = -3; p.shift[:] = 0          # a scale outside the shift-32 form: the window form on the two-SM kernel
+    _both_paths(p)
