@@ -61,7 +61,8 @@ typedef enum {
     I8_PATH_NONE = 0,       /* nothing launched (empty problem or error) */
     I8_PATH_GENERIC = 1,    /* one-thread-per-output kernel: any strides, any alignment */
     I8_PATH_TENSOR = 2,     /* TMA -> shared memory ring -> tcgen05.mma kind::i8 -> tensor memory -> epilogue */
-    I8_PATH_SMALL = 3       /* small-tile tensor path: resident B / paired 64x64 problems */
+    I8_PATH_SMALL = 3,      /* small-tile tensor path: paired 64x64 problems */
+    I8_PATH_TENSOR_2SM = 4  /* tensor path on clusters of two CTAs (tcgen05.mma.cta_group::2, 256 x 256 tiles) */
 } i8_path;
 
 /*
@@ -190,8 +191,9 @@ int i8ops_last_cuda_error(void);
 /* i8_path of the most recent compute call made by this thread. */
 int i8ops_last_path(void);
 
-/* Restrict dispatch: 0 = automatic (default), 1 = always the generic kernel, 2 = tensor paths whenever
- * their layout requirements hold (also for tiny problems).  Returns the previous setting. */
+/* Restrict dispatch: 0 = automatic (default), 1 = always the generic kernel, 2 = GEMMs take the two-SM tensor
+ * kernel whenever the layout allows the tensor path (also where its large tiles do not pay).  Returns the
+ * previous setting. */
 int i8ops_set_path(int mode);
 
 /* Upper limit, in milliseconds, for any single wait inside a kernel (default 2000). */

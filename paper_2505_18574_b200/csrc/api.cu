@@ -42,6 +42,7 @@ static int g_force_bn = -1;                      // tuning override from the env
 
 static thread_local int t_last_path = I8_PATH_NONE;
 static thread_local int t_last_cuda = 0;
+static thread_local bool t_used_two_sm = false;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -230,6 +231,9 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
     }
 }
 
+#ifndef I8_TC2_GROUP_M
+#define I8_TC2_GROUP_M 16     // tile rows walked together by neighbouring clusters (measured best of 2..32 on 8192^3)
+#endif
 // Two-SM kernel: 256 x 256 tiles, one cluster of two CTAs per tile.
 static int run_gemm_tc2(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                         const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
@@ -257,7 +261,7 @@ static int run_gemm_tc2(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8
     p.sched.m_tiles = (M + 255) / 256;
     p.sched.n_tiles = (N + TC2_BN - 1) / TC2_BN;
     p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
-    p.sched.group_m = 8;
+    p.sched.group_m = I8_TC2_GROUP_M;
     p.kl = KLoop{};
     p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);
     p.dev_status = ctx->dev_status;
@@ -274,8 +278,15 @@ static int run_gemm_tc2(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8
 static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
                        int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
-    if (g_tc2 && M >= 512 && N >= 512 && g_force_bn < 0)
-        return run_gemm_tc2(ctx, A, lda, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
+    {
+        // two-SM kernel: worth it once its 256 x 256 tiles fill at least half of the SM pairs (or when asked for)
+        const int64_t tiles2 = (int64_t)((M + 255) / 256) * ((N + 255) / 256);
+        const bool big = M >= 512 && N >= 512 && 4 * tiles2 >= ctx->sm_count;
+        if (g_force_bn < 0 && ((g_tc2 && big) || g_path_mode == 2)) {
+            t_used_two_sm = true;
+            return run_gemm_tc2(ctx, A, lda, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
+        }
+    }
     const int bn = choose_bn(M, N, (K + BK - 1) / BK, ctx->sm_count);
     CUtensorMap tmA;
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
@@ -408,8 +419,9 @@ int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_
     const bool tc_legal = K >= 1 && a_cs == 1 && b_rs == 1 && aligned16(A) && aligned16(B) && a_rs % 16 == 0 &&
                           b_cs % 16 == 0 && a_rs >= K && b_cs >= K;
     if (tc_legal && g_path_mode != 1) {
+        t_used_two_sm = false;
         rc = run_gemm_tc(ctx, A, a_rs, B, b_cs, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
-        if (rc == I8_OK) t_last_path = I8_PATH_TENSOR;
+        if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
         return rc;
     }
     GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, C, ldc, 0, bias, 0, mult, shift, per_channel, relu, 1, M, N, K, nullptr, 0, 0, 0};
@@ -434,8 +446,9 @@ int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, in
                           b_cs % 16 == 0 && a_rs >= K && b_cs >= K;
     if (tc_legal && g_path_mode != 1) {
         RawOut raw; raw.D = D; raw.ldd = ldd; raw.accumulate = accumulate ? 1 : 0;
+        t_used_two_sm = false;
         rc = run_gemm_tc(ctx, A, a_rs, B, b_cs, nullptr, 0, nullptr, nullptr, nullptr, 0, M, N, K, 0, st, raw);
-        if (rc == I8_OK) t_last_path = I8_PATH_TENSOR;
+        if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
         return rc;
     }
     GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, nullptr, 0, 0, nullptr, 0, nullptr, nullptr, 0, 0, 1, M, N, K,
@@ -495,8 +508,9 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
     if (g_path_mode != 1 && aligned16(x) && aligned16(w)) {
         if (R == 1 && S == 1 && stride_h == 1 && stride_w == 1 && pad_h == 0 && pad_w == 0 && C % 16 == 0) {
             // a 1x1 convolution is the GEMM [N*H*W, C] x [C, K]
+            t_used_two_sm = false;
             rc = run_gemm_tc(ctx, x, C, w, C, y, K, bias, mult, shift, per_channel, N * H * W, K, C, relu, st);
-            if (rc == I8_OK) t_last_path = I8_PATH_TENSOR;
+            if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
             return rc;
         }
         // im2col tensor maps: channel blocks of 32/64/128 bytes, box corners and tap offsets within the 4-D

@@ -16,15 +16,20 @@ def _auto_path():
     i8.set_path(0)
 
 
-def _both_paths(p, expect_tensor=True):
+TENSOR_PATHS = (2, 4)      # one-SM and two-SM tensor kernels
+
+
+def _both_paths(p, expect_tensor=True, two_sm=False):
     import paper_2505_18574_b200 as i8
     want = H.gemm_oracle(p)
-    i8.set_path(0)
+    i8.set_path(2 if two_sm else 0)
     got = H.gemm_gpu(p)
     path = i8.last_path()
     H.assert_same(got, want, f"{p.name} auto path={path}")
-    if expect_tensor:
-        assert path == i8.PATH_TENSOR, f"{p.name}: expected the tensor path, got {path}"
+    if two_sm:
+        assert path == i8.PATH_TENSOR_2SM, f"{p.name}: expected the two-SM kernel, got {path}"
+    elif expect_tensor:
+        assert path in TENSOR_PATHS, f"{p.name}: expected a tensor path, got {path}"
     i8.set_path(1)
     got = H.gemm_gpu(p)
     assert i8.last_path() == i8.PATH_GENERIC
@@ -98,7 +103,7 @@ def test_closed_forms_on_gpu():
         p = inputs.make_gemm(256, 128, K, 3, per_channel=0, relu=0, with_bias=False)
         p.A[:] = a; p.B[:] = b; p.mult[:] = mult; p.shift[:] = shift
         got = H.gemm_gpu(p)
-        assert i8.last_path() == i8.PATH_TENSOR
+        assert i8.last_path() in TENSOR_PATHS
         assert (got == expect).all(), (a, b, K, np.unique(got))
 
 
@@ -106,7 +111,7 @@ def test_config1a_full():
     p = inputs.config1(0)
     import paper_2505_18574_b200 as i8
     got = H.gemm_gpu(p)
-    assert i8.last_path() == i8.PATH_TENSOR
+    assert i8.last_path() == i8.PATH_TENSOR_2SM
     want = H.gemm_oracle(p)
     H.assert_same(got, want, p.name)
     H.not_degenerate(want)
@@ -118,7 +123,7 @@ def test_config1_large_sampled(j):
     import paper_2505_18574_b200 as i8
     p = inputs.config1(j)
     got = H.gemm_gpu(p)
-    assert i8.last_path() == i8.PATH_TENSOR
+    assert i8.last_path() == i8.PATH_TENSOR_2SM
     rng = np.random.default_rng(j)
     rows = np.unique(np.concatenate([rng.integers(0, p.M, size=500), [0, 1, 127, 128, p.M - 129, p.M - 128, p.M - 1]]))
     want = H.gemm_oracle_rows(p, rows)
@@ -168,7 +173,7 @@ def test_raw_accumulator_readout_and_split_k(M, N, K, ldd_pad):
         D = Dbuf[:, :N]
         i8.gemm_i8_raw(A, B.t(), D)
         assert i8.last_device_status() == 0
-        assert i8.last_path() == (i8.PATH_TENSOR if mode == 0 else i8.PATH_GENERIC)
+        assert i8.last_path() in (TENSOR_PATHS if mode == 0 else (i8.PATH_GENERIC,))
         H.assert_same(D.cpu().numpy(), want, f"raw mode {mode}")
         if ldd_pad:
             assert (Dbuf[:, N:] == 77).all()
@@ -181,14 +186,15 @@ def test_raw_accumulator_readout_and_split_k(M, N, K, ldd_pad):
     i8.set_path(0)
 
 
-@pytest.mark.parametrize("M,N,K", [(512, 512, 128), (513, 600, 1040), (1000, 520, 272), (640, 1300, 144), (769, 1025, 48), (2048, 1536, 4096)])
+@pytest.mark.parametrize("M,N,K", [(512, 512, 128), (513, 600, 1040), (1000, 520, 272), (640, 1300, 144), (769, 1025, 48), (2048, 1536, 4096),
+                                   (100, 300, 64), (256, 64, 96)])
 def test_two_sm_kernel_shapes(M, N, K):
     """Shapes with M, N >= 512 run on the two-SM (cta_group::2) kernel: ragged edges in M, N and K, both epilogue forms."""
     pad = (-K) % 16
     for per_channel, relu, shift_hi in ((1, 0, 22), (0, 1, 18)):
         p = inputs.make_gemm(M, N, K, 2000 + M + N + K, per_channel=per_channel, relu=relu, shift_lo=12, shift_hi=shift_hi,
                              lda_pad=pad, ldb_pad=pad, ldc_pad=16 * per_channel)
-        _both_paths(p)
+        _both_paths(p, two_sm=True)
     p = inputs.make_gemm(M, N, K, 7, per_channel=0, relu=0, lda_pad=pad, ldb_pad=pad)
     p.mult[:] = -3; p.shift[:] = 0          # a scale outside the shift-32 form: the window form on the two-SM kernel
-    _both_paths(p)
+    _both_paths(p, two_sm=True)

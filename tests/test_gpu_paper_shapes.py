@@ -15,7 +15,7 @@ def test_paper_gemm_shapes(i):
     p = inputs.sweep_gemm(i)
     i8.set_path(0)
     got = H.gemm_gpu(p)
-    assert i8.last_path() == i8.PATH_TENSOR
+    assert i8.last_path() in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM)
     if p.M * p.N * p.K <= 2 ** 36:
         want = H.gemm_oracle(p)
         H.assert_same(got, want, p.name)

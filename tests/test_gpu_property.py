@@ -34,6 +34,11 @@ def test_random_gemms(M, N, K16, seed, pads, relu, per_channel, with_bias, scale
     got = H.gemm_gpu(p)
     assert i8.last_path() == i8.PATH_TENSOR
     H.assert_same(got, want, f"{p.name} seed {seed} tensor")
+    i8.set_path(2)                                      # the same problem on the two-SM kernel
+    got = H.gemm_gpu(p)
+    assert i8.last_path() == i8.PATH_TENSOR_2SM
+    i8.set_path(0)
+    H.assert_same(got, want, f"{p.name} seed {seed} two-SM")
 
 
 @settings(max_examples=15, deadline=None, suppress_health_check=list(HealthCheck))
