@@ -279,9 +279,12 @@ static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_
                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
                        int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
     {
-        // two-SM kernel: worth it once its 256 x 256 tiles fill at least half of the SM pairs (or when asked for)
+        // two-SM kernel: its larger tiles and cluster set-up cost about 1.5 us more per launch, which pays once there
+        // is at least one full wave of 256 x 256 tiles and enough K per cluster (measured crossover: waves x K blocks ~ 48)
+        const int clusters = ctx->sm_count / 2;
         const int64_t tiles2 = (int64_t)((M + 255) / 256) * ((N + 255) / 256);
-        const bool big = M >= 512 && N >= 512 && 4 * tiles2 >= ctx->sm_count;
+        const int64_t waves2 = (tiles2 + clusters - 1) / clusters;
+        const bool big = tiles2 >= clusters && waves2 * ((K + BK - 1) / BK) >= 48;
         if (g_force_bn < 0 && ((g_tc2 && big) || g_path_mode == 2)) {
             t_used_two_sm = true;
             return run_gemm_tc2(ctx, A, lda, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
