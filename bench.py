@@ -147,7 +147,8 @@ def run_reference(args, rank, world):
     import oracle
     oracle.build()
     problems = [inputs.config1(j) for j in range(3)]
-    rows = {0: 512, 1: 128, 2: 256}     # per step: a bounded slab of each problem
+    rows = {0: 512, 1: 128, 2: 256}     # per step: a bounded slab of each problem (scaled down below for long runs)
+
     def step():
         macs = 0.0
         for j, p in enumerate(problems):
@@ -156,6 +157,15 @@ def run_reference(args, rank, world):
             oracle.gemm_i8(A, p.a_rs, 1, p.B, p.b_rs, p.b_cs, p.N, p.bias, p.mult, p.shift, p.per_channel, r, p.N, p.K, p.relu)
             macs += float(r) * p.N * p.K
         return macs
+
+    # keep the whole run to a couple of minutes: one calibration step, then shrink the slabs if K steps would take longer
+    t0 = time.perf_counter()
+    step()
+    t_base = time.perf_counter() - t0
+    budget_s = 100.0
+    if (args.steps + args.warmup) * t_base > budget_s:
+        f = max(budget_s / ((args.steps + args.warmup) * t_base), 1.0 / 32.0)
+        rows = {j: max(16, int(r * f) // 16 * 16) for j, r in rows.items()}
     for _ in range(args.warmup):
         step()
     t0 = time.perf_counter()
