@@ -12,7 +12,6 @@
 #include "../../include/i8ops.h"
 #include "batched_tc.cuh"
 #include "gemm_tc.cuh"
-#include "gemm_tc2.cuh"
 #include "generic.cuh"
 #include "mpc.cuh"
 
@@ -38,6 +37,7 @@ static int g_path_mode = 0;                      // 0 auto, 1 generic only, 2 te
 static uint64_t g_wait_limit_ns = 2000ull * 1000 * 1000;
 static int g_pdl = 1;                            // programmatic dependent launch (I8OPS_PDL=0 turns it off)
 static int g_tc2 = 1;                            // two-SM GEMM kernel for large shapes (I8OPS_TC2=0 turns it off)
+static int g_conv_two_sm = -1;                   // CTA pairs for convolutions: -1 by rule, 0 never, 1 always (I8OPS_CONV2SM)
 static int g_force_bn = -1;                      // tuning override from the environment (I8OPS_FORCE_BN)
 
 static thread_local int t_last_path = I8_PATH_NONE;
@@ -88,6 +88,8 @@ static int get_ctx(DeviceCtx** out) {
         }
         const char* bn = getenv("I8OPS_FORCE_BN");
         if (bn) g_force_bn = atoi(bn);
+        const char* c2 = getenv("I8OPS_CONV2SM");
+        if (c2) g_conv_two_sm = atoi(c2);
         const char* tc2 = getenv("I8OPS_TC2");
         if (tc2) g_tc2 = atoi(tc2);
         const char* pdl = getenv("I8OPS_PDL");
@@ -115,18 +117,29 @@ static int make_tmap(CUtensorMap* tm, const void* base, int rank, const uint64_t
 // Launch on `st`; with programmatic stream serialisation the kernel may be scheduled while its predecessor in
 // the stream drains (the kernels wait for their dependencies before touching global memory).
 template <typename... KArgs, typename... Args>
-static cudaError_t launch_kernel(void (*kern)(KArgs...), bool overlap, int grid, int block, size_t smem, cudaStream_t st,
-                                 Args&&... args) {
+static cudaError_t launch_kernel(void (*kern)(KArgs...), bool overlap, int cluster, int grid, int block, size_t smem,
+                                 cudaStream_t st, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (g_pdl && overlap) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        n++;
+    }
+    if (cluster > 1) {                      // CTA pairs: clusters of `cluster` consecutive CTAs
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cluster;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        n++;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = (g_pdl && overlap) ? 1 : 0;
+    cfg.numAttrs = n;
     return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
@@ -137,19 +150,21 @@ static CUtensorMapSwizzle swizzle_for(int cb) {
     return cb == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (cb == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
 }
 
-template <int BN, int STAGES, bool CONV, int EPI_WARPS, int NPROD>
+template <int BN, int STAGES, bool CONV, int EPI_WARPS, int NPROD, bool TWO_SM>
 static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUtensorMap& tmB, GemmTcParams& p,
                      cudaStream_t st) {
-    using L = TcSmem<BN, STAGES>;
-    auto kern = gemm_i8_tc_kernel<BN, STAGES, CONV, EPI_WARPS, NPROD>;
+    using L = TcSmem<BN, STAGES, TWO_SM>;
+    auto kern = gemm_i8_tc_kernel<BN, STAGES, CONV, EPI_WARPS, NPROD, TWO_SM>;
     if (!ctx->attr_set[slot]) {
         CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES));
         ctx->attr_set[slot] = true;
     }
-    const int grid = p.sched.num_tiles < ctx->sm_count ? p.sched.num_tiles : ctx->sm_count;
+    const int workers = TWO_SM ? ctx->sm_count / 2 : ctx->sm_count;          // CTAs, or CTA pairs
+    const int used = p.sched.num_tiles < workers ? p.sched.num_tiles : workers;
     // short kernels gain from overlapping their launch with the predecessor's tail; long ones do not need it
-    const bool overlap = 2.0 * p.M * p.N * p.K < 4e10;
-    CUDA_TRY(launch_kernel(kern, overlap, grid, 32 * (1 + NPROD) + 32 * EPI_WARPS, L::DYN_BYTES, st, tmA, tmB, p));
+    const bool overlap = !TWO_SM && 2.0 * p.M * p.N * p.K < 4e10;
+    CUDA_TRY(launch_kernel(kern, overlap, TWO_SM ? 2 : 1, TWO_SM ? 2 * used : used, 32 * (1 + NPROD) + 32 * EPI_WARPS, L::DYN_BYTES,
+                           st, tmA, tmB, p));
     return I8_OK;
 }
 
@@ -189,14 +204,18 @@ static int choose_bn(int M, int N, int num_kb, int sm_count) {
 // and the launch of the instance that matches the tile width.
 struct RawOut { int32_t* D = nullptr; int64_t ldd = 0; int accumulate = 0; };
 
-static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop& kl, int bn, const int8_t* B, int64_t ldb,
-                  int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
-                  int M, int N, int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
+static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA, const KLoop& kl, int bn, const int8_t* B,
+                  int64_t ldb, int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult, const int32_t* shift,
+                  int per_channel, int M, int N, int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
+    const int b_rows = two_sm ? bn / 2 : bn;           // rows of the B tile one CTA loads
+    const int tile_m = two_sm ? 2 * BM : BM;
+    // ring slots per instance (must match the launch table below)
+    const int stages = two_sm ? (bn == 256 ? 6 : 8) : (bn == 256 ? 4 : (bn == 128 ? 6 : 8));
     CUtensorMap tmB;
     {
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
         const uint64_t str[1] = {(uint64_t)ldb};
-        const uint32_t box[2] = {(uint32_t)kl.cb, (uint32_t)bn};
+        const uint32_t box[2] = {(uint32_t)kl.cb, (uint32_t)b_rows};
         int rc = make_tmap(&tmB, B, 2, dims, str, box, swizzle_for(kl.cb));
         if (rc) return rc;
     }
@@ -205,92 +224,54 @@ static int run_tc(DeviceCtx* ctx, bool conv, const CUtensorMap& tmA, const KLoop
     p.per_channel = per_channel; p.relu = relu; p.M = M; p.N = N; p.K = K;
     p.c_vec_ok = raw.D ? (aligned16(raw.D) && raw.ldd % 4 == 0) : (aligned16(C) && (ldc % 16 == 0));
     p.D = raw.D; p.ldd = raw.ldd; p.raw = raw.D ? 1 : 0; p.accumulate = raw.accumulate;
-    p.sched.m_tiles = (M + BM - 1) / BM;
+    p.sched.m_tiles = (M + tile_m - 1) / tile_m;
     p.sched.n_tiles = (N + bn - 1) / bn;
     p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
-    p.sched.group_m = 16;
+    p.sched.group_m = 16;                              // measured best of 2..32 on 8192^3 for the two-SM kernel
     p.kl = kl;
-    {
-        // resident B: one block column, and all of B's K blocks fit the ring's B region
-        const int stages = bn == 256 ? 4 : (bn == 128 ? 6 : 8);
-        p.kl.b_resident = (p.sched.n_tiles == 1 && (int64_t)kl.num_kblocks * bn * kl.cb <= (int64_t)stages * bn * BK) ? 1 : 0;
-    }
+    // resident B: one block column, and all of B's K blocks fit the ring's B region
+    p.kl.b_resident = (p.sched.n_tiles == 1 && (int64_t)kl.num_kblocks * b_rows * kl.cb <= (int64_t)stages * b_rows * BK) ? 1 : 0;
     p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);   // SM clock stays below 2 GHz: at least the asked time
     p.dev_status = ctx->dev_status;
+    if (two_sm) {
+        if (conv) {
+            switch (bn) {
+                case 256: return launch_tc<256, 6, true, 8, 2, true>(ctx, 8, tmA, tmB, p, st);
+                case 128: return launch_tc<128, 8, true, 8, 2, true>(ctx, 9, tmA, tmB, p, st);
+                default:  return launch_tc<64, 8, true, 8, 2, true>(ctx, 10, tmA, tmB, p, st);
+            }
+        }
+        return launch_tc<256, 6, false, 8, 1, true>(ctx, 7, tmA, tmB, p, st);
+    }
     if (conv) {
         switch (bn) {
-            case 256: return launch_tc<256, 4, true, 8, 2>(ctx, 3, tmA, tmB, p, st);
-            case 128: return launch_tc<128, 6, true, 8, 2>(ctx, 4, tmA, tmB, p, st);
-            default:  return launch_tc<64, 8, true, 8, 2>(ctx, 5, tmA, tmB, p, st);
+            case 256: return launch_tc<256, 4, true, 8, 2, false>(ctx, 3, tmA, tmB, p, st);
+            case 128: return launch_tc<128, 6, true, 8, 2, false>(ctx, 4, tmA, tmB, p, st);
+            default:  return launch_tc<64, 8, true, 8, 2, false>(ctx, 5, tmA, tmB, p, st);
         }
     }
     switch (bn) {
-        case 256: return launch_tc<256, 4, false, 8, 1>(ctx, 0, tmA, tmB, p, st);
-        case 128: return launch_tc<128, 6, false, 8, 1>(ctx, 1, tmA, tmB, p, st);
-        default:  return launch_tc<64, 8, false, 8, 1>(ctx, 2, tmA, tmB, p, st);
+        case 256: return launch_tc<256, 4, false, 8, 1, false>(ctx, 0, tmA, tmB, p, st);
+        case 128: return launch_tc<128, 6, false, 8, 1, false>(ctx, 1, tmA, tmB, p, st);
+        default:  return launch_tc<64, 8, false, 8, 1, false>(ctx, 2, tmA, tmB, p, st);
     }
-}
-
-#ifndef I8_TC2_GROUP_M
-#define I8_TC2_GROUP_M 16     // tile rows walked together by neighbouring clusters (measured best of 2..32 on 8192^3)
-#endif
-// Two-SM kernel: 256 x 256 tiles, one cluster of two CTAs per tile.
-static int run_gemm_tc2(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
-                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
-                        int K, int relu, cudaStream_t st, const RawOut& raw) {
-    CUtensorMap tmA, tmB;
-    {
-        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
-        const uint64_t str[1] = {(uint64_t)lda};
-        const uint32_t box[2] = {BK, BM};
-        int rc = make_tmap(&tmA, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
-        if (rc) return rc;
-    }
-    {
-        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
-        const uint64_t str[1] = {(uint64_t)ldb};
-        const uint32_t box[2] = {BK, TC2_BN / 2};
-        int rc = make_tmap(&tmB, B, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
-        if (rc) return rc;
-    }
-    GemmTcParams p;
-    p.C = C; p.ldc = ldc; p.bias = bias; p.mult = mult; p.shift = shift;
-    p.per_channel = per_channel; p.relu = relu; p.M = M; p.N = N; p.K = K;
-    p.c_vec_ok = raw.D ? (aligned16(raw.D) && raw.ldd % 4 == 0) : (aligned16(C) && (ldc % 16 == 0));
-    p.D = raw.D; p.ldd = raw.ldd; p.raw = raw.D ? 1 : 0; p.accumulate = raw.accumulate;
-    p.sched.m_tiles = (M + 255) / 256;
-    p.sched.n_tiles = (N + TC2_BN - 1) / TC2_BN;
-    p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
-    p.sched.group_m = I8_TC2_GROUP_M;
-    p.kl = KLoop{};
-    p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);
-    p.dev_status = ctx->dev_status;
-    if (!ctx->attr_set[7]) {
-        CUDA_TRY(cudaFuncSetAttribute(gemm_i8_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Tc2Smem::DYN_BYTES));
-        ctx->attr_set[7] = true;
-    }
-    int clusters = ctx->sm_count / 2;
-    if (p.sched.num_tiles < clusters) clusters = p.sched.num_tiles;
-    CUDA_TRY(launch_kernel(gemm_i8_tc2_kernel, false, 2 * clusters, TC2_THREADS, Tc2Smem::DYN_BYTES, st, tmA, tmB, p));
-    return I8_OK;
 }
 
 static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
                        int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
+    // two-SM kernel: its larger tiles and cluster set-up cost about 1.5 us more per launch, which pays once there
+    // is at least one full wave of 256 x 256 tiles and enough K per cluster (measured crossover: waves x K blocks ~ 48)
+    bool two_sm = false;
     {
-        // two-SM kernel: its larger tiles and cluster set-up cost about 1.5 us more per launch, which pays once there
-        // is at least one full wave of 256 x 256 tiles and enough K per cluster (measured crossover: waves x K blocks ~ 48)
         const int clusters = ctx->sm_count / 2;
         const int64_t tiles2 = (int64_t)((M + 255) / 256) * ((N + 255) / 256);
         const int64_t waves2 = (tiles2 + clusters - 1) / clusters;
         const bool big = tiles2 >= clusters && waves2 * ((K + BK - 1) / BK) >= 48;
-        if (g_force_bn < 0 && ((g_tc2 && big) || g_path_mode == 2)) {
-            t_used_two_sm = true;
-            return run_gemm_tc2(ctx, A, lda, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
-        }
+        two_sm = g_force_bn < 0 && ((g_tc2 && big) || g_path_mode == 2);
     }
-    const int bn = choose_bn(M, N, (K + BK - 1) / BK, ctx->sm_count);
+    t_used_two_sm = two_sm;
+    const int bn = two_sm ? 256 : choose_bn(M, N, (K + BK - 1) / BK, ctx->sm_count);
     CUtensorMap tmA;
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
     const uint64_t str[1] = {(uint64_t)lda};
@@ -301,7 +282,7 @@ static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_
     kl.cb = BK; kl.nsub = 1; kl.num_kblocks = (K + BK - 1) / BK;
     kl.num_iters = kl.num_kblocks;
     kl.mmas_last = ((K - (kl.num_iters - 1) * BK) + 31) / 32;
-    return run_tc(ctx, false, tmA, kl, bn, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
+    return run_tc(ctx, false, two_sm, tmA, kl, bn, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
 }
 
 // Implicit-GEMM convolution: A tiles come from an im2col-mode tensor map over the NHWC activations.
@@ -311,6 +292,16 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     const int cb = C % 128 == 0 ? 128 : (C % 64 == 0 ? 64 : 32);
     const int M = N * P * Q;
     const int bn = choose_bn(M, Kf, (R * S * C + BK - 1) / BK, ctx->sm_count);
+    // CTA pairs for convolutions: the same measured rule as for GEMMs (a full wave of 256-row tiles and enough K per
+    // cluster to amortise the pair's extra set-up), or asked for explicitly (path mode 2, I8OPS_CONV2SM=1)
+    bool two_sm = g_path_mode == 2 || g_conv_two_sm == 1;
+    if (g_tc2 && g_conv_two_sm != 0 && g_force_bn < 0) {
+        const int clusters = ctx->sm_count / 2;
+        const int64_t tiles2 = (int64_t)((M + 255) / 256) * ((Kf + bn - 1) / bn);
+        const int64_t waves2 = (tiles2 + clusters - 1) / clusters;
+        if (tiles2 >= clusters && waves2 * ((R * S * C + BK - 1) / BK) >= 48) two_sm = true;
+    }
+    t_used_two_sm = two_sm;
     CUtensorMap tmA;
     {
         const cuuint64_t gdim[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
@@ -332,7 +323,7 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     kl.mmas_last = (kl.num_kblocks - (kl.num_iters - 1) * kl.nsub) * (cb / 32);
     kl.stride_h = stride_h; kl.stride_w = stride_w; kl.pad_h = pad_h; kl.pad_w = pad_w;
     const int K = R * S * C;
-    return run_tc(ctx, true, tmA, kl, bn, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
+    return run_tc(ctx, true, two_sm, tmA, kl, bn, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
 }
 
 // Paired small-tile path: problems with M, N, K <= 64, two per MMA.
@@ -369,7 +360,7 @@ static int run_batched_pair(DeviceCtx* ctx, const int8_t* A, int64_t a_rs, int64
     }
     const int pairs = (batch + 1) / 2;
     const int grid = pairs < ctx->sm_count ? pairs : ctx->sm_count;
-    CUDA_TRY(launch_kernel(batched_pair_i8_kernel, true, grid, PAIR_THREADS, PairSmem::DYN_BYTES, st, tmA, tmB, p));
+    CUDA_TRY(launch_kernel(batched_pair_i8_kernel, true, 1, grid, PAIR_THREADS, PairSmem::DYN_BYTES, st, tmA, tmB, p));
     return I8_OK;
 }
 
@@ -521,9 +512,10 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
         const bool tc_legal = C % 32 == 0 && R <= 16 && S <= 16 && pad_h <= 16 && pad_w <= 16 && stride_h <= 8 &&
                               stride_w <= 8 && (int64_t)N * H * W * C >= 131072 && (int64_t)N * P * Q < (1ll << 31);
         if (tc_legal) {
+            t_used_two_sm = false;
             rc = run_conv_tc(ctx, x, w, y, bias, mult, shift, per_channel, N, H, W, C, K, R, S, P, Q, stride_h, stride_w,
                              pad_h, pad_w, relu, st);
-            if (rc == I8_OK) t_last_path = I8_PATH_TENSOR;
+            if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
             return rc;
         }
     }

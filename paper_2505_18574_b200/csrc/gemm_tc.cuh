@@ -12,6 +12,12 @@
 // matrix ever exists in memory.  A ring slot always holds 128 bytes of K per row, as 1, 2 or 4 sub-blocks
 // of cb = 128, 64 or 32 bytes (cb = the channel block; plain GEMMs use one 128-byte block).
 //
+// TWO_SM = true runs the same roles on clusters of two CTAs that share one 256 x BN tile through
+// tcgen05.mma.cta_group::2: each CTA holds 128 rows of A and BN / 2 rows of the B tile (a third less L2 and
+// shared-memory traffic per product at BN = 256), the even CTA's MMA warp issues for both tensor cores, TMA loads of
+// either CTA are counted on the even CTA's barriers, commits are multicast to both CTAs' barriers, and the odd CTA's
+// epilogue warps arrive remotely on the even CTA's accumulator-free barrier.  No load uses cluster multicast.
+//
 // The roles map onto the decoupled load / execute / store controllers of the accelerator that the paper
 // targets (Gemmini ISA description, Prompts appendix), and the two accumulators are the paper's
 // accumulator double-buffering (Code Examples appendix, the optimised 12544x64x256 GEMM), so that the
@@ -77,10 +83,11 @@ struct GemmTcParams {
     unsigned* dev_status;
 };
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, bool TWO_SM = false>
 struct TcSmem {
+    static constexpr int B_ROWS = TWO_SM ? BN / 2 : BN;        // a CTA of a pair holds half of the tile's B rows
     static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_BYTES = BN * BK;
+    static constexpr int B_BYTES = B_ROWS * BK;
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
     static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // 7 int32[BN] arrays of per-channel constants
@@ -167,11 +174,13 @@ __device__ __forceinline__ void store_raw_chunk(int32_t* drow, int n, int N, boo
     }
 }
 
-template <int BN, int STAGES, bool CONV, int EPI_WARPS, int NPROD>
+template <int BN, int STAGES, bool CONV, int EPI_WARPS, int NPROD, bool TWO_SM>
 __global__ void __launch_bounds__(32 * (1 + NPROD) + 32 * EPI_WARPS, 1)
 gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmTcParams p) {
-    using L = TcSmem<BN, STAGES>;
+    using L = TcSmem<BN, STAGES, TWO_SM>;
     constexpr int EPI_THREADS = 32 * EPI_WARPS;
+    constexpr int TILE_M = TWO_SM ? 2 * BM : BM;       // rows of one output tile (a CTA pair shares a 256-row tile)
+    constexpr int B_ROWS = L::B_ROWS;
     constexpr int NTHREADS = 32 * (1 + NPROD) + EPI_THREADS;
     constexpr int PROD2_WARP = 2 + EPI_WARPS;         // the optional second producer is the last warp
     static_assert(NPROD == 1 || NPROD == 2, "one or two producer warps");
@@ -207,6 +216,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
     const int lane = threadIdx.x & 31;
     const WaitEnv env{s_stop, p.dev_status, p.wait_limit_cycles};
+    // CTA pairs: rank 0 (even CTA) issues the MMAs; its full / accumulator-free / resident-B barriers serve both CTAs
+    const uint32_t rank = TWO_SM ? cluster_ctarank() : 0u;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) {
@@ -215,15 +226,21 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
         for (int b = 0; b < 2; b++) {
             mbar_init(bar_acc_full + 8 * b, 1);
-            mbar_init(bar_acc_empty + 8 * b, EPI_THREADS);
+            // one-SM: every epilogue thread arrives; pair: one lane of every epilogue warp of both CTAs
+            mbar_init(bar_acc_empty + 8 * b, TWO_SM ? 2 * EPI_WARPS : EPI_THREADS);
         }
         mbar_init(bar_bres, 1);
         *s_stop = 0;
         fence_barrier_init();
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(s_tmem)), L::TMEM_COLS);
-        tmem_relinquish();
+        if (TWO_SM) {
+            tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(s_tmem)), L::TMEM_COLS);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(const_cast<uint32_t*>(s_tmem)), L::TMEM_COLS);
+            tmem_relinquish();
+        }
     }
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmA);
@@ -235,7 +252,13 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // Set-up barrier.  The producer warp initialised the mbarriers itself and needs nothing from the others, so it
     // only signals and starts loading at once; everybody else waits for the barriers and the tensor-memory address.
     uint32_t tmem_base = 0;
-    if (warp == 0) {
+    if (TWO_SM) {
+        // both CTAs' barriers must exist before anything remote touches them
+        tc_fence_before();
+        cluster_sync_all();
+        tc_fence_after();
+        tmem_base = __shfl_sync(0xffffffffu, *s_tmem, 0);
+    } else if (warp == 0) {
         __syncwarp();
         named_barrier_arrive(15, NTHREADS);
     } else if (NPROD == 2 && warp == PROD2_WARP) {
@@ -249,7 +272,15 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
     const TileSched sched = p.sched;
     const KLoop kl = p.kl;
-    const uint32_t a_sub_bytes = BM * kl.cb, b_sub_bytes = BN * kl.cb;
+    const uint32_t a_sub_bytes = BM * kl.cb, b_sub_bytes = B_ROWS * kl.cb;
+    // persistent schedule: CTA (or CTA pair) w takes tiles w, w + W, w + 2W, ...
+    const int first_tile = TWO_SM ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int tile_step = TWO_SM ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    // barriers of the even CTA, as seen from this CTA (its own in the one-SM kernel)
+    const uint32_t full0 = TWO_SM ? map_to_cta(bar_full, 0) : bar_full;
+    const uint32_t bres0 = TWO_SM ? map_to_cta(bar_bres, 0) : bar_bres;
+    const uint32_t acc_empty0 = TWO_SM ? map_to_cta(bar_acc_empty, 0) : bar_acc_empty;
+    const uint32_t tx_mult = TWO_SM ? 2u : 1u;         // the even CTA's barriers count both CTAs' bytes
 
     if (warp == 0 || (NPROD == 2 && warp == PROD2_WARP)) {
         // ------------------------------------------------------------------ producer (whole warp loops, one lane issues)
@@ -261,20 +292,25 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         bool ok = true;
         const bool leader = elect_one();
         const bool bres = kl.b_resident != 0;
-        if (bres && pid == 0 && blockIdx.x < sched.num_tiles && leader) {
+        if (bres && pid == 0 && first_tile < sched.num_tiles && leader) {
             // the paper's "keep B resident" step: the whole (small) B operand is fetched once per CTA into the
             // region the ring would otherwise use for B, and only A streams
-            mbar_expect_tx(bar_bres, kl.num_kblocks * b_sub_bytes);
-            for (int kb = 0; kb < kl.num_kblocks; kb++) tma_load_2d(sB + kb * b_sub_bytes, &tmB, bar_bres, kb * kl.cb, 0);
+            if (rank == 0) mbar_expect_tx(bar_bres, tx_mult * kl.num_kblocks * b_sub_bytes);
+            for (int kb = 0; kb < kl.num_kblocks; kb++) {
+                if (TWO_SM) tma_load_2d_pair(sB + kb * b_sub_bytes, &tmB, bres0, kb * kl.cb, (int)rank * B_ROWS);
+                else tma_load_2d(sB + kb * b_sub_bytes, &tmB, bar_bres, kb * kl.cb, 0);
+            }
         }
         const uint32_t stage_tx = a_sub_bytes + (bres ? 0u : b_sub_bytes);
-        for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
+        for (int tile = first_tile; ok && tile < sched.num_tiles; tile += tile_step) {
             int m_blk, n_blk;
             sched.map(tile, m_blk, n_blk);
+            const int row_a = m_blk * TILE_M + (int)rank * BM;          // this CTA's first A row (output row / pixel)
+            const int row_b = n_blk * BN + (int)rank * B_ROWS;          // this CTA's first B row (output column)
             int w0 = 0, h0 = 0, img = 0;
             if (CONV) {
                 // first output pixel of the tile -> position of filter tap (0,0) in the input image
-                const int m0 = m_blk * BM;
+                const int m0 = row_a;
                 const int pq = kl.P * kl.Q;
                 img = fast_div(m0, pq, kl.inv_pq);
                 const int rem = m0 - img * pq;
@@ -293,27 +329,35 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     continue;
                 }
                 if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
-                const uint32_t full = bar_full + 8 * stage;
-                if (leader) mbar_expect_tx(full, nb * stage_tx);
+                const uint32_t full = full0 + 8 * stage;
+                if (leader && rank == 0) mbar_expect_tx(bar_full + 8 * stage, tx_mult * nb * stage_tx);
                 for (int j = 0; j < nb; j++, kbi++) {
                     const uint32_t dstA = sA + stage * L::A_BYTES + j * a_sub_bytes;
                     const uint32_t dstB = sB + stage * L::B_BYTES + j * b_sub_bytes;
                     if (CONV) {
-                        if (leader) tma_load_im2col_4d(dstA, &tmA, full, c_idx * kl.cb, w0, h0, img, (uint16_t)fs, (uint16_t)fr);
+                        if (leader) {
+                            if (TWO_SM) tma_load_im2col_4d_pair(dstA, &tmA, full, c_idx * kl.cb, w0, h0, img, (uint16_t)fs, (uint16_t)fr);
+                            else tma_load_im2col_4d(dstA, &tmA, full, c_idx * kl.cb, w0, h0, img, (uint16_t)fs, (uint16_t)fr);
+                        }
                         if (++c_idx == kl.cblocks) { c_idx = 0; if (++fs == kl.S) { fs = 0; ++fr; } }
-                    } else {
-                        if (leader) tma_load_2d(dstA, &tmA, full, kbi * BK, m_blk * BM);
+                    } else if (leader) {
+                        if (TWO_SM) tma_load_2d_pair(dstA, &tmA, full, kbi * BK, row_a);
+                        else tma_load_2d(dstA, &tmA, full, kbi * BK, row_a);
                     }
-                    if (leader && !bres) tma_load_2d(dstB, &tmB, full, kbi * kl.cb, n_blk * BN);
+                    if (leader && !bres) {
+                        if (TWO_SM) tma_load_2d_pair(dstB, &tmB, full, kbi * kl.cb, row_b);
+                        else tma_load_2d(dstB, &tmB, full, kbi * kl.cb, row_b);
+                    }
                 }
                 issued |= 1u << stage;
                 issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
                 if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
         }
-        if (*s_stop) {
-            // stopping early: let every copy this warp started land before the CTA retires
-            if (bres && pid == 0 && blockIdx.x < sched.num_tiles && !mbar_wait_drain(bar_bres, 0, p.wait_limit_cycles))
+        if (*s_stop && rank == 0) {
+            // stopping early: let every copy this warp started land before the CTA retires (in a pair the even CTA's
+            // barriers also count the odd CTA's copies, and the closing cluster barrier keeps the odd CTA alive meanwhile)
+            if (bres && pid == 0 && first_tile < sched.num_tiles && !mbar_wait_drain(bar_bres, 0, p.wait_limit_cycles))
                 atomicCAS(p.dev_status, 0u, (unsigned)DEV_TIMEOUT_DRAIN);
             for (int s = 0; s < STAGES; s++)
                 if (issued & (1u << s))
@@ -323,7 +367,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (whole warp loops, one lane issues)
-        constexpr uint32_t idesc = make_idesc_i8(BM, BN, 0, 0);
+        constexpr uint32_t idesc = make_idesc_i8(TILE_M, BN, 0, 0);   // a pair's instruction spans both CTAs' rows
         // K-major operands: rows cb bytes apart, swizzled over cb bytes, 8-row groups 8*cb bytes apart;
         // a 32-byte step along K inside a swizzle row is a plain address offset.
         const uint64_t swz = kl.cb == 128 ? SWZ_128B : (kl.cb == 64 ? SWZ_64B : SWZ_32B);
@@ -346,8 +390,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         bool ok = true;
         const bool bres = kl.b_resident != 0;
         const uint32_t b_iter_units = (kl.nsub * b_sub_bytes) >> 4;   // resident B: descriptor units per ring slot's worth of K
-        if (bres && blockIdx.x < sched.num_tiles) ok = mbar_wait_warp(bar_bres, 0, env, DEV_TIMEOUT_MMA_FULL);
-        for (int tile = blockIdx.x; ok && tile < sched.num_tiles; tile += gridDim.x) {
+        if (rank != 0) ok = false;                       // in a pair only the even CTA issues
+        if (ok && bres && first_tile < sched.num_tiles) ok = mbar_wait_warp(bar_bres, 0, env, DEV_TIMEOUT_MMA_FULL);
+        for (int tile = first_tile; ok && tile < sched.num_tiles; tile += tile_step) {
             if (!mbar_wait_warp(bar_acc_empty + 8 * ab, acc_phase ^ 1, env, DEV_TIMEOUT_MMA_ACC)) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + ab * BN;
@@ -365,17 +410,25 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const uint32_t b0 = b_base + (bres ? it * b_iter_units : stage * (L::B_BYTES >> 4));
 #pragma unroll
                     for (int i = 0; i < 4; i++)
-                        if (i < nm)
-                            mma_i8_ss(d_tmem, desc_hi | (uint64_t)(a0 + offA[i]), desc_hi | (uint64_t)(b0 + offB[i]), idesc,
-                                      (it | i) != 0 ? 1u : 0u);
-                    tc_commit(bar_empty + 8 * stage);    // slot reusable once these MMAs have read it
+                        if (i < nm) {
+                            if (TWO_SM) mma_i8_ss_pair(d_tmem, desc_hi | (uint64_t)(a0 + offA[i]), desc_hi | (uint64_t)(b0 + offB[i]), idesc,
+                                                       (it | i) != 0 ? 1u : 0u);
+                            else mma_i8_ss(d_tmem, desc_hi | (uint64_t)(a0 + offA[i]), desc_hi | (uint64_t)(b0 + offB[i]), idesc,
+                                           (it | i) != 0 ? 1u : 0u);
+                        }
+                    // slot reusable once these MMAs have read it (in a pair: in both CTAs)
+                    if (TWO_SM) tc_commit_pair(bar_empty + 8 * stage);
+                    else tc_commit(bar_empty + 8 * stage);
                 }
                 ready = __all_sync(0xffffffffu, peek);
                 stage = nstage;
                 phase = nphase;
             }
             if (!ok) break;
-            if (leader) tc_commit(bar_acc_full + 8 * ab);   // accumulator complete
+            if (leader) {                                    // accumulator complete (both halves in a pair)
+                if (TWO_SM) tc_commit_pair(bar_acc_full + 8 * ab);
+                else tc_commit(bar_acc_full + 8 * ab);
+            }
             ab ^= 1;
             if (ab == 0) acc_phase ^= 1;
         }
@@ -391,7 +444,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int32_t rb[ONE_CHUNK ? 32 : 1], rm[ONE_CHUNK ? 32 : 1];   // register copy of the constants (ONE_CHUNK only)
         uint32_t acc_phase = 0;
         bool dead = false;
-        for (int tile = blockIdx.x; tile < sched.num_tiles; tile += gridDim.x) {
+        for (int tile = first_tile; tile < sched.num_tiles; tile += tile_step) {
             int m_blk, n_blk;
             sched.map(tile, m_blk, n_blk);
             const int n0 = n_blk * BN;
@@ -427,7 +480,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (!dead) dead = !__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * ab, acc_phase, env, DEV_TIMEOUT_EPILOGUE));
             if (dead) continue;
             tc_fence_after();
-            const int row = m_blk * BM + quarter * 32 + lane;
+            const int row = m_blk * TILE_M + (int)rank * BM + quarter * 32 + lane;
             int8_t* crow = p.C + (int64_t)row * p.ldc;
             const uint32_t t0 = tmem_base + ab * BN + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
@@ -459,17 +512,31 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 if (row < p.M) store_row_chunk(crow, n, p.N, p.c_vec_ok != 0, out);
             }
             tc_fence_before();
-            mbar_arrive(bar_acc_empty + 8 * ab);
+            if (TWO_SM) {
+                // one lane per warp tells the even CTA that this warp's share of the accumulator is free
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(acc_empty0 + 8 * ab);
+            } else {
+                mbar_arrive(bar_acc_empty + 8 * ab);
+            }
             ab ^= 1;
             if (ab == 0) acc_phase ^= 1;
         }
     }
 
     tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        tmem_dealloc(tmem_base, L::TMEM_COLS);
+    if (TWO_SM) {
+        cluster_sync_all();        // neither CTA leaves or frees tensor memory while the other still works
+        if (warp == 1) {
+            tc_fence_after();
+            tmem_dealloc_pair(tmem_base, L::TMEM_COLS);
+        }
+    } else {
+        __syncthreads();
+        if (warp == 1) {
+            tc_fence_after();
+            tmem_dealloc(tmem_base, L::TMEM_COLS);
+        }
     }
 }
 

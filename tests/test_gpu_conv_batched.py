@@ -24,7 +24,7 @@ def _conv_both(p, expect_tensor=None):
     path = i8.last_path()
     H.assert_same(got, want, f"{p.name} auto path={path}")
     if expect_tensor is not None:
-        assert (path == i8.PATH_TENSOR) == expect_tensor, f"{p.name}: path {path}"
+        assert (path in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM)) == expect_tensor, f"{p.name}: path {path}"
     i8.set_path(1)
     got = H.conv_gpu(p)
     assert i8.last_path() == i8.PATH_GENERIC
@@ -59,6 +59,21 @@ def test_conv_tensor_path(N, H_, W, C, K, R, S, st, pad):
     assert N * H_ * W * C >= 131072
     p = inputs.make_conv(N, H_, W, C, K, R, S, st, pad, 500 + N + H_ + C + K)
     _conv_both(p, expect_tensor=True)
+
+
+@pytest.mark.parametrize("N,H_,W,C,K,R,S,st,pad", [
+    (4, 28, 28, 64, 64, 3, 3, 1, 1), (8, 12, 12, 128, 64, 3, 3, 2, 1), (4, 15, 13, 192, 80, 3, 3, 2, 1), (8, 24, 24, 32, 48, 3, 3, 1, 1),
+    (6, 14, 14, 256, 256, 3, 3, 1, 1), (5, 17, 17, 128, 136, 3, 3, 1, 0), (2, 40, 36, 64, 192, 3, 3, 1, 1), (3, 30, 30, 64, 64, 7, 7, 2, 3),
+])
+def test_conv_cta_pair_kernel(N, H_, W, C, K, R, S, st, pad):
+    """The same convolutions forced onto clusters of two CTAs (cta_group::2, im2col loads counted on the even CTA)."""
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_conv(N, H_, W, C, K, R, S, st, pad, 900 + N + H_ + C + K)
+    want = H.conv_oracle(p)
+    i8.set_path(2)
+    got = H.conv_gpu(p)
+    assert i8.last_path() == i8.PATH_TENSOR_2SM
+    H.assert_same(got, want, p.name + " two-SM")
 
 
 def test_conv_delta_filter_on_gpu():

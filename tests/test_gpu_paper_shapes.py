@@ -33,7 +33,7 @@ def test_paper_conv_shapes(i):
     p = inputs.sweep_conv(i)
     i8.set_path(0)
     got = H.conv_gpu(p)
-    assert i8.last_path() == i8.PATH_TENSOR
+    assert i8.last_path() in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM)
     if p.N * p.P * p.Q * p.K * p.R * p.S * p.C <= 2 ** 34:
         want = H.conv_oracle(p)
         H.assert_same(got, want, p.name)
