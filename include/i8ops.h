@@ -132,7 +132,8 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y,
  * Host-buffer variants: every pointer is HOST memory (pinned memory makes the copies asynchronous).
  * The call copies the operands to a device workspace that the library keeps per device (grown with
  * cudaMalloc when a larger problem arrives, never shrunk), runs the same kernels, copies the result
- * back and synchronises `stream` before returning.  They also check every shift (I8_ERR_RANGE).
+ * back and synchronises `stream` before returning.  Problems with 2048 rows or more are cut into row chunks whose
+ * copy-in, kernel and copy-out overlap on three streams (two of them internal).  They also check every shift (I8_ERR_RANGE).
  * Tight layouts only: A row-major [M][K], B column-major (K contiguous, [N][K]), C row-major [M][N].
  */
 int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C,

@@ -29,6 +29,8 @@ struct DeviceCtx {
     bool attr_set[16] = {};           // dynamic shared-memory opt-in done, per kernel instance
     void* ws = nullptr;               // workspace of the host-buffer variants
     size_t ws_bytes = 0;
+    cudaStream_t s_in = nullptr, s_out = nullptr;   // copy streams of the host-buffer variants
+    cudaEvent_t ev[2 * 8 + 2] = {};                 // chunk hand-over events (up to 8 row chunks)
 };
 
 static DeviceCtx g_ctx[MAX_DEVICES];
@@ -560,16 +562,61 @@ int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C, const int32_t* bia
     int32_t* dbias = (int32_t*)(base + szA + szB + szC);
     int32_t* dmult = (int32_t*)((uint8_t*)dbias + szV);
     int32_t* dshift = (int32_t*)((uint8_t*)dmult + szV);
-    if (K > 0) {
-        CUDA_TRY(cudaMemcpyAsync(dA, A, (size_t)M * K, cudaMemcpyHostToDevice, st));
-        CUDA_TRY(cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, st));
+    // Row chunks are pipelined over three streams: copy-in of chunk i+1, the kernel on chunk i and copy-out of chunk i-1
+    // overlap (the two copy directions use separate DMA engines), so the host link is busy in both directions.
+    const int nchunks = (K > 0 && M >= 2048) ? (M >= 8192 ? 8 : 4) : 1;
+    if (nchunks > 1 && !ctx->s_in) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!ctx->s_in) {
+            CUDA_TRY(cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking));
+            for (auto& e : ctx->ev) CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+            CUDA_TRY(cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking));
+        }
     }
-    if (bias) CUDA_TRY(cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, st));
-    CUDA_TRY(cudaMemcpyAsync(dmult, mult, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
-    CUDA_TRY(cudaMemcpyAsync(dshift, shift, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
-    rc = gemm_i8(dA, K, 1, dB, 1, K, dC, N, bias ? dbias : nullptr, dmult, dshift, per_channel, M, N, K, relu, stream);
-    if (rc) return rc;
-    CUDA_TRY(cudaMemcpyAsync(C, dC, (size_t)M * N, cudaMemcpyDeviceToHost, st));
+    if (nchunks == 1) {
+        if (K > 0) {
+            CUDA_TRY(cudaMemcpyAsync(dA, A, (size_t)M * K, cudaMemcpyHostToDevice, st));
+            CUDA_TRY(cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, st));
+        }
+        if (bias) CUDA_TRY(cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, st));
+        CUDA_TRY(cudaMemcpyAsync(dmult, mult, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
+        CUDA_TRY(cudaMemcpyAsync(dshift, shift, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
+        rc = gemm_i8(dA, K, 1, dB, 1, K, dC, N, bias ? dbias : nullptr, dmult, dshift, per_channel, M, N, K, relu, stream);
+        if (rc) return rc;
+        CUDA_TRY(cudaMemcpyAsync(C, dC, (size_t)M * N, cudaMemcpyDeviceToHost, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+        return I8_OK;
+    }
+    cudaEvent_t* ev_in = ctx->ev;            // [i]: chunk i of A (and, for i = 0, B and the vectors) is on the device
+    cudaEvent_t* ev_k = ctx->ev + 8;         // [i]: the kernel of chunk i is done
+    cudaEvent_t ev_start = ctx->ev[16], ev_done = ctx->ev[17];
+    CUDA_TRY(cudaEventRecord(ev_start, st)); // the copy streams start after whatever the caller queued on `stream`
+    CUDA_TRY(cudaStreamWaitEvent(ctx->s_in, ev_start, 0));
+    CUDA_TRY(cudaStreamWaitEvent(ctx->s_out, ev_start, 0));
+    CUDA_TRY(cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, ctx->s_in));
+    if (bias) CUDA_TRY(cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, ctx->s_in));
+    CUDA_TRY(cudaMemcpyAsync(dmult, mult, (size_t)nq * 4, cudaMemcpyHostToDevice, ctx->s_in));
+    CUDA_TRY(cudaMemcpyAsync(dshift, shift, (size_t)nq * 4, cudaMemcpyHostToDevice, ctx->s_in));
+    const int rows_per = (((M + nchunks - 1) / nchunks) + 255) / 256 * 256;
+    int used = 0;
+    for (int i = 0; i < nchunks; i++) {
+        const int r0 = i * rows_per;
+        if (r0 >= M) break;
+        const int rows = M - r0 < rows_per ? M - r0 : rows_per;
+        CUDA_TRY(cudaMemcpyAsync(dA + (size_t)r0 * K, A + (size_t)r0 * K, (size_t)rows * K, cudaMemcpyHostToDevice, ctx->s_in));
+        CUDA_TRY(cudaEventRecord(ev_in[i], ctx->s_in));
+        CUDA_TRY(cudaStreamWaitEvent(st, ev_in[i], 0));
+        rc = gemm_i8(dA + (size_t)r0 * K, K, 1, dB, 1, K, dC + (size_t)r0 * N, N, bias ? dbias : nullptr, dmult, dshift, per_channel,
+                     rows, N, K, relu, stream);
+        if (rc) return rc;
+        CUDA_TRY(cudaEventRecord(ev_k[i], st));
+        CUDA_TRY(cudaStreamWaitEvent(ctx->s_out, ev_k[i], 0));
+        CUDA_TRY(cudaMemcpyAsync(C + (size_t)r0 * N, dC + (size_t)r0 * N, (size_t)rows * N, cudaMemcpyDeviceToHost, ctx->s_out));
+        used++;
+    }
+    (void)used;
+    CUDA_TRY(cudaEventRecord(ev_done, ctx->s_out));
+    CUDA_TRY(cudaStreamWaitEvent(st, ev_done, 0));
     CUDA_TRY(cudaStreamSynchronize(st));
     return I8_OK;
 }

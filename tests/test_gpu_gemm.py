@@ -198,3 +198,22 @@ def test_two_sm_kernel_shapes(M, N, K):
     p = inputs.make_gemm(M, N, K, 7, per_channel=0, relu=0, lda_pad=pad, ldb_pad=pad)
     p.mult[:] = -3; p.shift[:] = 0          # a scale outside the shift-32 form: the window form on the two-SM kernel
     _both_paths(p, two_sm=True)
+
+
+@pytest.mark.parametrize("M,N,K,pinned", [(300, 200, 112, False), (2048, 512, 256, True), (5000, 384, 160, True), (8192, 256, 128, False)])
+def test_host_buffer_variant(M, N, K, pinned):
+    """gemm_i8_host: host buffers in, host buffer out (row chunks pipelined over three streams for M >= 2048)."""
+    import torch
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_gemm(M, N, K, 31 + M, per_channel=1, relu=1, shift_lo=12, shift_hi=20)
+    want = H.gemm_oracle(p)
+    mk = (lambda a: torch.from_numpy(a).pin_memory()) if pinned else (lambda a: torch.from_numpy(a))
+    A, B, bias, mult, shift = mk(p.A), mk(p.B), mk(p.bias), mk(p.mult), mk(p.shift)
+    C = torch.full((M, N), 0x5A, dtype=torch.int8)
+    if pinned:
+        C = C.pin_memory()
+    for _ in range(2):                               # twice: the second call reuses the workspace, streams and events
+        C.fill_(0x5A)
+        i8.gemm_i8_host(A, B, C, bias, mult, shift, 1, 1)
+        H.assert_same(C.numpy(), want, p.name + " host variant")
+    assert i8.last_device_status() == 0
