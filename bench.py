@@ -35,7 +35,7 @@ WORKLOAD = "config1: int8 GEMM (4096,4096,4096)+(8192,8192,8192)+(16384,4096,819
 NOMINAL_INT8_OVER_BF16 = 2.0          # dense 4.5 POPS int8 vs 2.25 PFLOP/s bf16
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
-NCU_STEP_TRAFFIC_BYTES = 656990322   # dram__bytes_read.sum + dram__bytes_write.sum over the step's three launches
+NCU_STEP_TRAFFIC_BYTES = 653448448   # dram__bytes_read.sum + dram__bytes_write.sum over the step's three launches
 
 
 def measured_peaks():
@@ -341,7 +341,7 @@ def main():
                              "so each problem's tiles are evicted before its next launch",
                        "per_problem_ms": {p.name: per_problem_ms[j] for j, p in enumerate(problems)},
                        "per_problem_tops": {p.name: gemm_ops(p) / (per_problem_ms[j] * 1e-3) / 1e12 for j, p in enumerate(problems)}},
-            "roofline": {"bound": "tensor", "kernel": "gemm_i8_tc2_kernel (two-SM, 256x256 tiles, cta_group::2)", "achieved": achieved, "peak": peak_int8,
+            "roofline": {"bound": "tensor", "kernel": "gemm_i8_tc_kernel<256,6,0,8,1,1> (CTA pairs, 256x256 tiles, cta_group::2)", "achieved": achieved, "peak": peak_int8,
                          "unit": "TFLOP/s", "frac": achieved / peak_int8, "traffic": NCU_STEP_TRAFFIC_BYTES,
                          "traffic_note": "DRAM bytes read+written by one step (one launch of each problem), ncu launch list in "
                                          "profiles/bench_config1_launch_list.txt; algorithmic bytes per step 4.87e8",
