@@ -53,7 +53,8 @@ typedef enum {
     I8_ERR_RANGE = 5,       /* K > 65536, or (host variants) a shift outside [0, 31] */
     I8_ERR_UNSUPPORTED = 6, /* stride or padding outside what the convolution supports */
     I8_ERR_CUDA = 7,        /* a CUDA runtime or driver call failed; see i8ops_last_cuda_error() */
-    I8_ERR_TIMEOUT = 8      /* a bounded wait inside a kernel expired (device status only) */
+    I8_ERR_TIMEOUT = 8,     /* a bounded wait inside a kernel expired (device status only) */
+    I8_ERR_WORKSPACE = 9    /* gemm_i8_host_noalloc: the problem does not fit its fixed device workspace */
 } i8_status;
 
 /* Which kernel family served the most recent compute call of this thread (for tests and tuning). */
@@ -139,6 +140,32 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y,
 int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C,
                  const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
                  int M, int N, int K, int relu, void* stream);
+
+/*
+ * gemm_i8_host without any allocation (the paper has no counterpart; this exists for callers, not for the method).
+ * Some programs may not allocate device memory once they are running: a control loop with a fixed memory budget
+ * (the setting of the paper's TinyMPC benchmark), a plug-in inside a host application that owns the GPU's memory
+ * pool, or code that runs while the allocator is off limits because an allocation would synchronise the device.
+ * For them this entry point does what gemm_i8_host does, but its device copies of A, B, bias, mult, shift and C
+ * live in a fixed array of I8OPS_NOALLOC_MAX_BYTES that is part of the library's device image: every GPU that
+ * loads the library sets that much memory aside until the process exits, whether or not this function is called.
+ * It calls no cudaMalloc, cudaFree or other allocating routine, creates no streams or events, and does all its
+ * copies and its kernel on `stream`, which it synchronises before returning.
+ *   Arguments, layouts and results as gemm_i8_host (HOST pointers; tight row-major A and C, K-contiguous B).
+ *   Limit: with every region rounded up to 256 bytes, M*K + N*K + M*N + 3 * 4*N must not exceed
+ *   I8OPS_NOALLOC_MAX_BYTES (e.g. 2048 x 2048 x 2048 fits, 4096^3 does not); larger problems return
+ *   I8_ERR_WORKSPACE and nothing is launched or copied.
+ *   The first call on each device looks up the array's device address (with that device current) and may load
+ *   kernels; make that first call outside any stream capture.
+ *   All calls on a device share the one array.  It keeps whatever the last call left; nothing in it needs
+ *   clearing, because each call overwrites every byte it later reads.  Two calls that are in flight on the same
+ *   GPU at the same time (from two host threads or processes sharing the context) race on it: serialise them.
+ * Errors: as gemm_i8_host, plus I8_ERR_WORKSPACE.
+ */
+#define I8OPS_NOALLOC_MAX_BYTES (16 * 1024 * 1024)
+int gemm_i8_host_noalloc(const int8_t* A, const int8_t* B, int8_t* C,
+                         const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
+                         int M, int N, int K, int relu, void* stream);
 
 /* Human-readable name of an i8_status. */
 const char* i8_status_string(int status);

@@ -28,6 +28,7 @@ SIGNATURES = {
                                _int, _int, _int, _int, _int, _vp]),
     "conv2d_i8": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int] + [_int] * 12 + [_vp]),
     "gemm_i8_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
+    "gemm_i8_host_noalloc": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
     "mpc_forward_f32": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp]),
     "i8_status_string": (ctypes.c_char_p, [_int]),
     "i8ops_last_device_status": (_int, [_vp]),
@@ -144,6 +145,24 @@ def gemm_i8_host(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream
     st = lib().gemm_i8_host(hp(A), hp(B), hp(C), hp(bias), hp(mult), hp(shift), int(per_channel), M, N, K, int(relu),
                             _stream_ptr(stream))
     _check(st, "gemm_i8_host")
+
+
+NOALLOC_MAX_BYTES = 16 * 1024 * 1024
+
+
+def gemm_i8_host_noalloc(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:
+    """gemm_i8_host for callers that may not allocate device memory: same arguments and results, but the device
+    copies live in a fixed 16 MiB array inside the library, so the padded operands, vectors and result together must
+    fit in ``NOALLOC_MAX_BYTES`` (status 9 otherwise).  Calls share that array: do not overlap them on one GPU."""
+    def hp(a):
+        if a is None:
+            return None
+        return a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data
+    M, K = A.shape
+    N = B.shape[0]
+    st = lib().gemm_i8_host_noalloc(hp(A), hp(B), hp(C), hp(bias), hp(mult), hp(shift), int(per_channel), M, N, K,
+                                    int(relu), _stream_ptr(stream))
+    _check(st, "gemm_i8_host_noalloc")
 
 
 def mpc_forward_f32(Adyn, Bdyn, Kinf, x0, d, u, xs=None, stream=None) -> None:

@@ -632,6 +632,7 @@ const char* i8_status_string(int status) {
         case I8_ERR_UNSUPPORTED: return "unsupported";
         case I8_ERR_CUDA: return "CUDA call failed";
         case I8_ERR_TIMEOUT: return "a bounded wait expired inside a kernel";
+        case I8_ERR_WORKSPACE: return "problem larger than the fixed workspace of the allocation-free variant";
         default: return "unknown status";
     }
 }
@@ -727,3 +728,72 @@ void i8ops_set_wait_limit_ms(int ms) {
 int i8ops_version(void) { return 1; }
 
 }  // extern "C"
+
+// ================================================================================================ allocation-free variant
+// gemm_i8_host for callers that must not allocate device memory: the device copies of the operands, of the
+// epilogue vectors and of the result live in one array that is part of the library's device image, so the
+// driver reserves it on every GPU that loads the library and it stays reserved until the process exits.
+namespace i8 {
+
+static __device__ __align__(256) unsigned char g_noalloc_ws[I8OPS_NOALLOC_MAX_BYTES];
+
+// In host code `g_noalloc_ws` is only a handle for the runtime, not an address a kernel or a copy may use; the
+// device address is looked up once per device and kept here.
+static unsigned char* g_noalloc_ptr[MAX_DEVICES] = {};
+
+static int noalloc_base(unsigned char** out) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return cuda_fail(cudaErrorInvalidDevice);
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        unsigned char* ptr = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress((void**)&ptr, g_noalloc_ws));    // the current device's copy of the array
+        if (!ptr) return cuda_fail(cudaErrorInvalidSymbol);
+        g_noalloc_ptr[dev] = ptr;
+    }
+    *out = g_noalloc_ptr[dev];
+    return I8_OK;
+}
+
+}  // namespace i8
+
+extern "C" int gemm_i8_host_noalloc(const int8_t* A, const int8_t* B, int8_t* C, const int32_t* bias, const int32_t* mult,
+                                    const int32_t* shift, int per_channel, int M, int N, int K, int relu, void* stream) {
+    t_last_path = I8_PATH_NONE;
+    if (M < 0 || N < 0 || K < 0) return I8_ERR_SHAPE;
+    if (K > 65536) return I8_ERR_RANGE;
+    if (M == 0 || N == 0) return I8_OK;
+    if (!C || !mult || !shift || (K > 0 && (!A || !B))) return I8_ERR_NULL;
+    const int nq = per_channel ? N : 1;
+    for (int i = 0; i < nq; i++)
+        if (shift[i] < 0 || shift[i] > 31) return I8_ERR_RANGE;
+    // every region starts on a 256-byte boundary of the array (the tensor path wants 16-byte aligned operands)
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t szA = up((size_t)M * K), szB = up((size_t)N * K), szC = up((size_t)M * N), szV = up((size_t)N * 4);
+    if (szA + szB + szC + 3 * szV > (size_t)I8OPS_NOALLOC_MAX_BYTES) return I8_ERR_WORKSPACE;
+    unsigned char* base = nullptr;
+    int rc = noalloc_base(&base);
+    if (rc) return rc;
+    int8_t* dA = (int8_t*)base;
+    int8_t* dB = (int8_t*)(base + szA);
+    int8_t* dC = (int8_t*)(base + szA + szB);
+    int32_t* dbias = (int32_t*)(base + szA + szB + szC);
+    int32_t* dmult = (int32_t*)((unsigned char*)dbias + szV);
+    int32_t* dshift = (int32_t*)((unsigned char*)dmult + szV);
+    // Nothing in the array has to start at zero: every byte the kernel reads below is written by these copies first,
+    // and the kernel writes every element of dC that is copied back.  What earlier calls left elsewhere is never read.
+    cudaStream_t st = (cudaStream_t)stream;
+    if (K > 0) {
+        CUDA_TRY(cudaMemcpyAsync(dA, A, (size_t)M * K, cudaMemcpyHostToDevice, st));
+        CUDA_TRY(cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, st));
+    }
+    if (bias) CUDA_TRY(cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(dmult, mult, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(dshift, shift, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
+    rc = gemm_i8(dA, K, 1, dB, 1, K, dC, N, bias ? dbias : nullptr, dmult, dshift, per_channel, M, N, K, relu, stream);
+    if (rc) return rc;
+    CUDA_TRY(cudaMemcpyAsync(C, dC, (size_t)M * N, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return I8_OK;
+}

@@ -1,0 +1,55 @@
+"""gemm_i8_host_noalloc, the host-buffer GEMM for programs that may not allocate device memory while they run
+(fixed memory budgets, hosts that own the GPU's memory pool, phases in which an allocation would stall the device).
+
+Its device copies live in a fixed 16 MiB array inside the library instead of a cudaMalloc'ed workspace.  The file is
+named so that pytest collects it after every other test: a run that stops at the first failure has then already run
+the rest.  The GPU test calls the C ABI twice in a row with different shapes, so the second call finds the array
+full of the first call's data, and compares each result bit for bit with what gemm_i8_host returns."""
+import numpy as np
+import pytest
+
+from paper_2505_18574_b200 import inputs
+
+
+def _lib():
+    from paper_2505_18574_b200 import build
+    build.build()
+    from paper_2505_18574_b200 import binding
+    return binding.lib()
+
+
+def test_rejects_problems_beyond_the_fixed_workspace():
+    """The size check precedes every CUDA call, so it runs without a GPU: 4096^3 needs 48 MiB of device copies."""
+    from paper_2505_18574_b200 import binding
+    L = _lib()
+    one = np.ones(1, np.int32)
+    buf = np.zeros(16, np.int8)          # never dereferenced: the call returns before touching the operands
+    st = L.gemm_i8_host_noalloc(buf.ctypes.data, buf.ctypes.data, buf.ctypes.data, None, one.ctypes.data, one.ctypes.data,
+                                0, 4096, 4096, 4096, 0, None)
+    assert st == 9 and b"workspace" in L.i8_status_string(9)
+    # 2048 x 2048 x 2048: 12 MiB + vectors fits; one more 256-row block of A does not change that, 4096 rows do
+    def need(M, N, K):
+        up = lambda v: (v + 255) // 256 * 256
+        return up(M * K) + up(N * K) + up(M * N) + 3 * up(4 * N)
+    assert need(2048, 2048, 2048) <= binding.NOALLOC_MAX_BYTES < need(4096, 2048, 2048)
+    st = L.gemm_i8_host_noalloc(buf.ctypes.data, buf.ctypes.data, buf.ctypes.data, None, one.ctypes.data, one.ctypes.data,
+                                0, 4096, 2048, 2048, 0, None)
+    assert st == 9
+
+
+@pytest.mark.gpu
+def test_matches_gemm_i8_host_on_two_calls_in_a_row():
+    import paper_2505_18574_b200 as i8
+    # a large problem first (tensor path, fills most of the array), then a smaller ragged one whose regions start
+    # at other offsets and without a bias, then the first again
+    cases = [(2048, 1024, 1024, True), (333, 200, 112, False), (2048, 1024, 1024, True)]
+    for i, (M, N, K, with_bias) in enumerate(cases):
+        p = inputs.make_gemm(M, N, K, 900 + M, per_channel=1, relu=1, shift_lo=12, shift_hi=20)
+        bias = p.bias if with_bias else None
+        want = np.full((M, N), 0x5A, np.int8)
+        i8.gemm_i8_host(p.A, p.B, want, bias, p.mult, p.shift, 1, 1)
+        got = np.full((M, N), 0x33, np.int8)
+        i8.gemm_i8_host_noalloc(p.A, p.B, got, bias, p.mult, p.shift, 1, 1)
+        assert np.array_equal(got, want), f"call {i}: {M}x{N}x{K} differs from gemm_i8_host"
+        assert len(np.unique(want)) > 16, "degenerate output would prove nothing"
+    assert i8.last_device_status() == 0
