@@ -97,6 +97,25 @@ __device__ __forceinline__ int32_t requant_shift32(int32_t acc, int32_t bias, in
     return (int32_t)(uint32_t)(p >> 32);
 }
 
+// Folded shift-32 form.  Because (acc + bias) * m2 + 2^31 = acc * m2 + (bias * m2 + 2^31), the bias can ride in the
+// 64-bit addend c = bias * m2 + 2^31 of the one widening multiply-add: |acc * m2| <= 2^62 and |c| <= 2^62 + 2^31, and
+// their sum is the in-range value above, so nothing wraps.  ReLU then has to move behind the scale, which is exact
+// whenever m2 >= 0: for t = acc + bias < 0 the scaled value floor((t * m2 + 2^31) / 2^32) is <= 0 and becomes 0 either
+// way, for t >= 0 it is unchanged.  The saturating pack keeps signs, so that late ReLU is "clear the negative bytes" of
+// the packed word (relu_s8x4): two instructions per four outputs instead of one max per output.
+__device__ __forceinline__ long long make_fold_addend(int32_t bias, int32_t m2) {
+    return (long long)bias * (long long)m2 + (1ll << 31);
+}
+__device__ __forceinline__ int32_t requant_fold(int32_t acc, int32_t m2, long long c) {
+    return (int32_t)(uint32_t)((unsigned long long)((long long)acc * (long long)m2 + c) >> 32);
+}
+// max(x, 0) on four packed signed bytes: prmt with selector bit 3 set replicates a byte's sign bit over the byte.
+__device__ __forceinline__ uint32_t relu_s8x4(uint32_t x) {
+    uint32_t neg;
+    asm("prmt.b32 %0, %1, %1, 0xba98;" : "=r"(neg) : "r"(x));
+    return x & ~neg;
+}
+
 // Saturate four 32-bit values to int8 and pack them, v0 in the lowest byte.
 // cvt.pack.sat.s8.s32.b32 d, a, b, c  gives  d = (c << 16) | (sat8(a) << 8) | sat8(b).
 __device__ __forceinline__ uint32_t pack_sat4(int32_t v0, int32_t v1, int32_t v2, int32_t v3) {

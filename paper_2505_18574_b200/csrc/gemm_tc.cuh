@@ -90,8 +90,8 @@ struct TcSmem {
     static constexpr int B_BYTES = B_ROWS * BK;
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-    static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // 7 int32[BN] arrays of per-channel constants
-    static constexpr int OFF_BAR = OFF_CONST + 7 * BN * 4;           // full[S], empty[S], acc_full[2], acc_empty[2], b_resident
+    static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // 7 int32[BN] arrays and one int64[BN] array of per-channel constants
+    static constexpr int OFF_BAR = OFF_CONST + 9 * BN * 4;           // full[S], empty[S], acc_full[2], acc_empty[2], b_resident
     static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 5) * 8;  // tensor-memory base, stop flag
     static constexpr int TOTAL = OFF_MISC + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;                   // slack to align the base to 1024 bytes
@@ -132,16 +132,29 @@ __device__ __forceinline__ void epilogue_chunk_shift32(const int32_t (&v)[32], c
     }
 }
 
-// The same with the 32 columns' constants already in registers (tiles whose warps keep a fixed column range).
+// Folded form: the bias rides in the 64-bit addend, ReLU is applied to the packed bytes (needs m2 >= 0 under ReLU).
 template <bool RELU>
-__device__ __forceinline__ void epilogue_chunk_shift32_regs(const int32_t (&v)[32], const int32_t (&rb)[32], const int32_t (&rm)[32],
-                                                            uint32_t (&out)[8]) {
+__device__ __forceinline__ void epilogue_chunk_fold(const int32_t (&v)[32], const int32_t* s_m2, const long long* s_c64, int c0,
+                                                    uint32_t (&out)[8]) {
 #pragma unroll
-    for (int j = 0; j < 8; j++)
-        out[j] = pack_sat4(requant_shift32<RELU>(v[4 * j + 0], rb[4 * j + 0], rm[4 * j + 0]),
-                           requant_shift32<RELU>(v[4 * j + 1], rb[4 * j + 1], rm[4 * j + 1]),
-                           requant_shift32<RELU>(v[4 * j + 2], rb[4 * j + 2], rm[4 * j + 2]),
-                           requant_shift32<RELU>(v[4 * j + 3], rb[4 * j + 3], rm[4 * j + 3]));
+    for (int j = 0; j < 8; j++) {
+        const int4 m2 = *reinterpret_cast<const int4*>(s_m2 + c0 + 4 * j);
+        const longlong2 ca = *reinterpret_cast<const longlong2*>(s_c64 + c0 + 4 * j);
+        const longlong2 cb = *reinterpret_cast<const longlong2*>(s_c64 + c0 + 4 * j + 2);
+        const uint32_t pk = pack_sat4(requant_fold(v[4 * j + 0], m2.x, ca.x), requant_fold(v[4 * j + 1], m2.y, ca.y),
+                                      requant_fold(v[4 * j + 2], m2.z, cb.x), requant_fold(v[4 * j + 3], m2.w, cb.y));
+        out[j] = RELU ? relu_s8x4(pk) : pk;
+    }
+}
+template <bool RELU>
+__device__ __forceinline__ void epilogue_chunk_fold_regs(const int32_t (&v)[32], const int32_t (&rm)[32], const long long (&rc)[32],
+                                                         uint32_t (&out)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+        const uint32_t pk = pack_sat4(requant_fold(v[4 * j + 0], rm[4 * j + 0], rc[4 * j + 0]), requant_fold(v[4 * j + 1], rm[4 * j + 1], rc[4 * j + 1]),
+                                      requant_fold(v[4 * j + 2], rm[4 * j + 2], rc[4 * j + 2]), requant_fold(v[4 * j + 3], rm[4 * j + 3], rc[4 * j + 3]));
+        out[j] = RELU ? relu_s8x4(pk) : pk;
+    }
 }
 
 // Store one thread's 32 output bytes (columns n .. n+31 of one row).
@@ -204,6 +217,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     int32_t* s_mult = s_hi + BN;
     int32_t* s_shift = s_mult + BN;
     int32_t* s_rnd = s_shift + BN;
+    long long* s_c64 = reinterpret_cast<long long*>(s_rnd + BN);     // folded form: bias * m2 + 2^31 (8-byte aligned: BN is even)
     const uint32_t bar_full = sbase + L::OFF_BAR;
     const uint32_t bar_empty = bar_full + STAGES * 8;
     const uint32_t bar_acc_full = bar_empty + STAGES * 8;
@@ -440,8 +454,10 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int cgroup = (warp - 2) >> 2;             // which share of the columns this warp handles
         int ab = 0, cached_n_blk = -1;
         bool shift32 = false;                           // every channel of the cached block admits the shift-32 form
+        bool fold = false;                              // ... and the folded form (under ReLU: no negative multiplier)
         constexpr bool ONE_CHUNK = COLS_PER_GROUP == 32;
-        int32_t rb[ONE_CHUNK ? 32 : 1], rm[ONE_CHUNK ? 32 : 1];   // register copy of the constants (ONE_CHUNK only)
+        int32_t rm[ONE_CHUNK ? 32 : 1];                 // register copy of the constants (ONE_CHUNK only)
+        long long rc[ONE_CHUNK ? 32 : 1];
         uint32_t acc_phase = 0;
         bool dead = false;
         for (int tile = first_tile; tile < sched.num_tiles; tile += tile_step) {
@@ -451,7 +467,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (n_blk != cached_n_blk) {
                 // new block column: rebuild the per-channel constants (before waiting, so this overlaps the main loop)
                 named_barrier(1, EPI_THREADS);            // nobody still reads the previous column's constants
-                bool all32 = true;
+                bool all32 = true, allfold = true;
                 for (int c = etid; c < BN; c += EPI_THREADS) {
                     const int n = n0 + c;
                     int32_t bias = 0, mult = 0, shift = 0;
@@ -464,15 +480,19 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     s_bias[c] = bias; s_lo[c] = cc.lo; s_hi[c] = cc.hi;
                     s_mult[c] = cc.mult; s_shift[c] = cc.shift; s_rnd[c] = cc.rnd;
                     int32_t m2;
-                    all32 = make_shift32_mult(mult, shift, m2) && all32;
+                    const bool ok32 = make_shift32_mult(mult, shift, m2);
+                    all32 = ok32 && all32;
+                    allfold = allfold && ok32 && (!p.relu || m2 >= 0);
                     s_m2[c] = m2;
+                    s_c64[c] = make_fold_addend(bias, m2);
                 }
                 cached_n_blk = n_blk;
                 shift32 = named_barrier_and(2, EPI_THREADS, all32);
-                if constexpr (ONE_CHUNK) if (shift32) {
+                fold = named_barrier_and(3, EPI_THREADS, allfold);
+                if constexpr (ONE_CHUNK) if (fold) {
                     // this warp's 32 columns are the same for every tile of the block column: keep them in registers
 #pragma unroll
-                    for (int j = 0; j < 32; j++) { rb[j] = s_bias[cgroup * 32 + j]; rm[j] = s_m2[cgroup * 32 + j]; }
+                    for (int j = 0; j < 32; j++) { rm[j] = s_m2[cgroup * 32 + j]; rc[j] = s_c64[cgroup * 32 + j]; }
                 }
             }
             // A warp whose wait expired stays in the loop without touching the accumulators, so that the barriers
@@ -498,14 +518,18 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     continue;
                 }
                 uint32_t out[8];
-                if (shift32) {
+                if (fold) {
                     if constexpr (ONE_CHUNK) {
-                        if (p.relu) epilogue_chunk_shift32_regs<true>(v, rb, rm, out);
-                        else epilogue_chunk_shift32_regs<false>(v, rb, rm, out);
+                        if (p.relu) epilogue_chunk_fold_regs<true>(v, rm, rc, out);
+                        else epilogue_chunk_fold_regs<false>(v, rm, rc, out);
                     } else {
-                        if (p.relu) epilogue_chunk_shift32<true>(v, s_bias, s_m2, c0, out);
-                        else epilogue_chunk_shift32<false>(v, s_bias, s_m2, c0, out);
+                        if (p.relu) epilogue_chunk_fold<true>(v, s_m2, s_c64, c0, out);
+                        else epilogue_chunk_fold<false>(v, s_m2, s_c64, c0, out);
                     }
+                } else if (shift32) {
+                    // ReLU with a negative multiplier somewhere in the block column: ReLU must stay ahead of the scale
+                    if (p.relu) epilogue_chunk_shift32<true>(v, s_bias, s_m2, c0, out);
+                    else epilogue_chunk_shift32<false>(v, s_bias, s_m2, c0, out);
                 } else {
                     epilogue_chunk(v, s_bias, s_lo, s_hi, s_mult, s_shift, s_rnd, c0, out);
                 }
