@@ -63,7 +63,8 @@ typedef enum {
     I8_PATH_GENERIC = 1,    /* one-thread-per-output kernel: any strides, any alignment */
     I8_PATH_TENSOR = 2,     /* TMA -> shared memory ring -> tcgen05.mma kind::i8 -> tensor memory -> epilogue */
     I8_PATH_SMALL = 3,      /* small-tile tensor path: paired 64x64 problems */
-    I8_PATH_TENSOR_2SM = 4  /* tensor path on clusters of two CTAs (tcgen05.mma.cta_group::2, 256 x 256 tiles) */
+    I8_PATH_TENSOR_2SM = 4, /* tensor path on clusters of two CTAs (tcgen05.mma.cta_group::2, 256 x 256 tiles) */
+    I8_PATH_CONV_SLAB = 5   /* stride-1 convolution with the input slab resident in shared memory and reused across taps */
 } i8_path;
 
 /*
@@ -219,9 +220,10 @@ int i8ops_last_cuda_error(void);
 /* i8_path of the most recent compute call made by this thread. */
 int i8ops_last_path(void);
 
-/* Restrict dispatch: 0 = automatic (default), 1 = always the generic kernel, 2 = GEMMs take the two-SM tensor
- * kernel whenever the layout allows the tensor path (also where its large tiles do not pay).  Returns the
- * previous setting. */
+/* Restrict dispatch: 0 = automatic (default), 1 = always the generic kernel, 2 = GEMMs and convolutions take the
+ * two-SM tensor kernel whenever the layout allows the tensor path (also where its large tiles do not pay),
+ * 3 = automatic, but stride-1 convolutions stay on the implicit-GEMM kernel instead of the slab kernel.
+ * Returns the previous setting. */
 int i8ops_set_path(int mode);
 
 /* Upper limit, in milliseconds, for any single wait inside a kernel (default 2000). */

@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libi8ops.so")
 _lib = None
 
-PATH_NONE, PATH_GENERIC, PATH_TENSOR, PATH_SMALL, PATH_TENSOR_2SM = 0, 1, 2, 3, 4
+PATH_NONE, PATH_GENERIC, PATH_TENSOR, PATH_SMALL, PATH_TENSOR_2SM, PATH_CONV_SLAB = 0, 1, 2, 3, 4, 5
 
 _vp = ctypes.c_void_p
 _i64 = ctypes.c_int64

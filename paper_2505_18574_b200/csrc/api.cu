@@ -11,6 +11,7 @@
 
 #include "../../include/i8ops.h"
 #include "batched_tc.cuh"
+#include "conv_slab.cuh"
 #include "gemm_tc.cuh"
 #include "generic.cuh"
 #include "mpc.cuh"
@@ -35,12 +36,13 @@ struct DeviceCtx {
 
 static DeviceCtx g_ctx[MAX_DEVICES];
 static std::mutex g_mutex;
-static int g_path_mode = 0;                      // 0 auto, 1 generic only, 2 tensor whenever legal
+static int g_path_mode = 0;                      // 0 auto, 1 generic only, 2 two-SM tensor kernel whenever legal, 3 auto without the slab convolution
 static uint64_t g_wait_limit_ns = 2000ull * 1000 * 1000;
 static int g_pdl = 1;                            // programmatic dependent launch (I8OPS_PDL=0 turns it off)
 static int g_tc2 = 1;                            // two-SM GEMM kernel for large shapes (I8OPS_TC2=0 turns it off)
 static int g_conv_two_sm = -1;                   // CTA pairs for convolutions: -1 by rule, 0 never, 1 always (I8OPS_CONV2SM)
 static int g_force_bn = -1;                      // tuning override from the environment (I8OPS_FORCE_BN)
+static int g_slab = 1;                           // slab-resident stride-1 convolution kernel (I8OPS_SLAB=0 turns it off)
 
 static thread_local int t_last_path = I8_PATH_NONE;
 static thread_local int t_last_cuda = 0;
@@ -94,6 +96,8 @@ static int get_ctx(DeviceCtx** out) {
         if (c2) g_conv_two_sm = atoi(c2);
         const char* tc2 = getenv("I8OPS_TC2");
         if (tc2) g_tc2 = atoi(tc2);
+        const char* slab = getenv("I8OPS_SLAB");
+        if (slab) g_slab = atoi(slab);
         const char* pdl = getenv("I8OPS_PDL");
         if (pdl) g_pdl = atoi(pdl);
         c.ready = true;
@@ -328,6 +332,75 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     return run_tc(ctx, true, two_sm, tmA, kl, bn, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
 }
 
+// Slab-resident stride-1 convolution (conv_slab.cuh): plan and launch.  Returns I8_ERR_UNSUPPORTED, launching nothing,
+// when the layer does not fit the kernel (the caller then takes the implicit-GEMM path).
+static int run_conv_slab(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, const int32_t* mult,
+                         const int32_t* shift, int per_channel, int N, int H, int W, int C, int Kf, int R, int S, int P, int Q,
+                         int pad_h, int pad_w, int relu, cudaStream_t st) {
+    const int Wp = W + 2 * pad_w;
+    if (C % 32 != 0 || Wp > BM || Kf > 128 || R * S > 49 || Q < 1 || P < 1) return I8_ERR_UNSUPPORTED;
+    const int TH = BM / Wp;
+    const int slab_rows = TH + R - 1;
+    if (slab_rows > 256 || 2 * TH * Q < BM) return I8_ERR_UNSUPPORTED;        // at least half of the 128 lanes must be real outputs
+    const int bn = Kf <= 64 ? 64 : 128;
+    const int cb = C % 128 == 0 ? 128 : (C % 64 == 0 ? 64 : 32);
+    const int cblocks = C / cb;
+    const int64_t tiles_per_img = (P + TH - 1) / TH;
+    if ((int64_t)N * tiles_per_img >= (1ll << 30)) return I8_ERR_UNSUPPORTED;
+    auto up1k = [](int64_t v) { return (v + 1023) & ~(int64_t)1023; };
+    const int64_t slab_tx = (int64_t)cb * Wp * slab_rows;
+    const int64_t reach = (int64_t)(BM + (R - 1) * Wp + S - 1) * cb;          // furthest byte any tap's 128 rows touch
+    const int64_t stage_bytes = up1k(slab_tx > reach ? slab_tx : reach);
+    const int64_t w_bytes = (int64_t)R * S * C * bn;                           // resident filter bank, zero rows up to bn
+    const int64_t fixed = up1k(w_bytes) + 9 * bn * 4 + (2 * SLAB_MAX_STAGES + 5) * 8 + 16;
+    const int64_t budget = 227 * 1024 - 1024;
+    int64_t stages = (budget - fixed) / stage_bytes;
+    if (stages > SLAB_MAX_STAGES) stages = SLAB_MAX_STAGES;
+    if (stages < 2) return I8_ERR_UNSUPPORTED;
+    CUtensorMap tmX, tmW;
+    {
+        const uint64_t dims[4] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+        const uint64_t str[3] = {(uint64_t)C, (uint64_t)W * C, (uint64_t)H * W * C};
+        const uint32_t box[4] = {(uint32_t)cb, (uint32_t)Wp, (uint32_t)slab_rows, 1};
+        int rc = make_tmap(&tmX, x, 4, dims, str, box, swizzle_for(cb));
+        if (rc) return rc;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)R * S * C, (uint64_t)Kf};
+        const uint64_t str[1] = {(uint64_t)R * S * C};
+        const uint32_t box[2] = {(uint32_t)cb, (uint32_t)bn};
+        int rc = make_tmap(&tmW, w, 2, dims, str, box, swizzle_for(cb));
+        if (rc) return rc;
+    }
+    ConvSlabParams p;
+    p.y = y; p.bias = bias; p.mult = mult; p.shift = shift; p.per_channel = per_channel; p.relu = relu;
+    p.Kf = Kf; p.P = P; p.Q = Q; p.R = R; p.S = S; p.Wp = Wp; p.TH = TH; p.pad_h = pad_h; p.pad_w = pad_w;
+    p.cb = cb; p.cblocks = cblocks;
+    p.tiles_per_img = (int)tiles_per_img; p.num_tiles = (int)(N * tiles_per_img);
+    p.inv_tpi = tiles_per_img == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)tiles_per_img);
+    p.inv_wp = Wp == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)Wp);
+    p.slab_tx_bytes = (int)slab_tx; p.stage_bytes = (int)stage_bytes; p.stages = (int)stages;
+    p.off_b = (int)(stages * stage_bytes);
+    p.off_const = p.off_b + (int)up1k(w_bytes);
+    p.off_bar = p.off_const + 9 * bn * 4;
+    p.y_vec_ok = aligned16(y) && Kf % 16 == 0;
+    p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);
+    p.dev_status = ctx->dev_status;
+    const size_t smem = (size_t)p.off_bar + (2 * SLAB_MAX_STAGES + 5) * 8 + 16 + 1024;
+    const int grid = p.num_tiles < ctx->sm_count ? p.num_tiles : ctx->sm_count;
+    // 3 x 3 filters get the instance whose issue loop is unrolled over the nine taps
+    void (*kern)(CUtensorMap, CUtensorMap, ConvSlabParams);
+    int slot;
+    if (R == 3 && S == 3) { kern = bn == 64 ? conv_slab_i8_kernel<64, 9> : conv_slab_i8_kernel<128, 9>; slot = bn == 64 ? 11 : 12; }
+    else { kern = bn == 64 ? conv_slab_i8_kernel<64, 0> : conv_slab_i8_kernel<128, 0>; slot = bn == 64 ? 13 : 14; }
+    if (!ctx->attr_set[slot]) {
+        CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        ctx->attr_set[slot] = true;
+    }
+    CUDA_TRY(launch_kernel(kern, true, 1, grid, SLAB_THREADS, smem, st, tmX, tmW, p));
+    return I8_OK;
+}
+
 // Paired small-tile path: problems with M, N, K <= 64, two per MMA.
 static int run_batched_pair(DeviceCtx* ctx, const int8_t* A, int64_t a_rs, int64_t a_bs, const int8_t* B, int64_t b_ld,
                             int64_t b_bs, int b_mn_major, int8_t* C, int64_t ldc, int64_t c_bs, const int32_t* bias,
@@ -508,6 +581,12 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
             rc = run_gemm_tc(ctx, x, C, w, C, y, K, bias, mult, shift, per_channel, N * H * W, K, C, relu, st);
             if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
             return rc;
+        }
+        if (g_slab && g_path_mode == 0 && stride_h == 1 && stride_w == 1 && (int64_t)N * P * Q < (1ll << 31)) {
+            // few filters and a narrow image: keep the input slab in shared memory and reuse it across the filter taps
+            rc = run_conv_slab(ctx, x, w, y, bias, mult, shift, per_channel, N, H, W, C, K, R, S, P, Q, pad_h, pad_w, relu, st);
+            if (rc == I8_OK) { t_last_path = I8_PATH_CONV_SLAB; return rc; }
+            if (rc != I8_ERR_UNSUPPORTED) return rc;
         }
         // im2col tensor maps: channel blocks of 32/64/128 bytes, box corners and tap offsets within the 4-D
         // encoding's ranges, traversal strides up to 8; activation tensors below 128 KiB stay on the generic kernel
@@ -716,7 +795,7 @@ int i8ops_last_path(void) { return t_last_path; }
 
 int i8ops_set_path(int mode) {
     const int prev = g_path_mode;
-    if (mode >= 0 && mode <= 2) g_path_mode = mode;
+    if (mode >= 0 && mode <= 3) g_path_mode = mode;
     return prev;
 }
 

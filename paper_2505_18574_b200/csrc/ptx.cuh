@@ -216,6 +216,16 @@ __device__ __forceinline__ void mma_i8_ss(uint32_t tmem_d, uint64_t adesc, uint6
         : "memory");
 }
 
+// The same with accumulation always on: no predicate to compute (the compiler folds the comparison to "true").
+__device__ __forceinline__ void mma_i8_ss_acc(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc)
+        : "memory");
+}
+
 // Instruction descriptor for kind::i8: int32 accumulator, signed int8 A and B, dense.
 //   [4,6) D format (2 = s32)   [7,10) A format (1 = s8)   [10,13) B format (1 = s8)
 //   [15] A is MN-major   [16] B is MN-major   [17,23) N >> 3   [24,29) M >> 4

@@ -24,7 +24,12 @@ def _conv_both(p, expect_tensor=None):
     path = i8.last_path()
     H.assert_same(got, want, f"{p.name} auto path={path}")
     if expect_tensor is not None:
-        assert (path in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM)) == expect_tensor, f"{p.name}: path {path}"
+        assert (path in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM, i8.PATH_CONV_SLAB)) == expect_tensor, f"{p.name}: path {path}"
+    if path == i8.PATH_CONV_SLAB:
+        i8.set_path(3)                                   # the same layer without the slab kernel
+        got = H.conv_gpu(p)
+        assert i8.last_path() != i8.PATH_CONV_SLAB, f"{p.name}: path {i8.last_path()}"
+        H.assert_same(got, want, f"{p.name} implicit GEMM (or generic, for small activations)")
     i8.set_path(1)
     got = H.conv_gpu(p)
     assert i8.last_path() == i8.PATH_GENERIC
@@ -81,17 +86,53 @@ def test_conv_delta_filter_on_gpu():
     import paper_2505_18574_b200 as i8
     p = inputs.make_conv(24, 9, 10, 64, 64, 3, 3, 1, 1, 5, per_channel=0, relu=0, with_bias=False, act_lo=-100, act_hi=101)
     p.mult[:] = 1; p.shift[:] = 0
-    for (r, s) in [(0, 0), (1, 1), (2, 0), (1, 2)]:
+    for (r, s, mode) in [(0, 0, 0), (1, 1, 0), (2, 0, 0), (1, 2, 0), (0, 2, 3), (2, 1, 3)]:
         p.w[:] = 0
         for k in range(64):
             p.w[k, r, s, (k + 3) % 64] = 1
+        i8.set_path(mode)
         got = H.conv_gpu(p)
-        assert i8.last_path() == i8.PATH_TENSOR
+        assert i8.last_path() == (i8.PATH_CONV_SLAB if mode == 0 else i8.PATH_TENSOR)
         for pp in range(p.P):
             for q in range(p.Q):
                 h = pp - 1 + r; w = q - 1 + s
                 want = p.x[:, h, w, :][:, [(k + 3) % 64 for k in range(64)]] if (0 <= h < 9 and 0 <= w < 10) else 0
                 assert np.array_equal(got[:, pp, q, :], np.broadcast_to(want, (24, 64))), (r, s, pp, q)
+
+
+@pytest.mark.parametrize("N,H_,W,C,K,R,S,pad", [
+    (3, 56, 56, 64, 64, 3, 3, (1, 1)),      # the 56 x 56 x 64 layer: two output rows per tile, 64-byte channel block
+    (5, 14, 14, 128, 128, 3, 3, (1, 1)),    # eight rows per tile, 128-byte channel block, 128 filters
+    (3, 14, 14, 256, 48, 3, 3, (1, 1)),     # two 128-byte channel blocks per tile
+    (4, 27, 31, 32, 40, 3, 3, (1, 1)),      # 32-byte block, ragged filter count, odd extents (row count not a multiple of the tile)
+    (2, 20, 100, 64, 64, 3, 3, (1, 1)),     # one row per tile (raster width 102)
+    (3, 19, 23, 96, 40, 5, 5, (2, 2)),      # 5 x 5 filter, three 32-byte blocks
+    (2, 33, 40, 64, 24, 3, 3, (0, 0)),      # no padding: output smaller than the input
+    (2, 30, 30, 32, 64, 7, 7, (3, 3)),      # 7 x 7 filter
+    (3, 18, 25, 128, 64, 3, 5, (1, 2)),     # rectangular filter with matching padding
+    (2, 24, 24, 64, 64, 3, 3, (2, 0)),      # unequal padding: taller output, narrower output
+    (1, 9, 62, 96, 8, 1, 3, (0, 1)),        # 1 x 3 filter, 8 filters
+    (7, 12, 12, 64, 64, 3, 3, (1, 1)),      # nine of the twelve rows in one tile, three in the next
+    (40, 28, 28, 64, 64, 3, 3, (1, 1)),     # 280 tiles: both issuers of every CTA take a turn
+])
+def test_conv_slab_kernel(N, H_, W, C, K, R, S, pad):
+    """Stride-1 layers with few filters run on the slab kernel (input rows resident in shared memory, taps read
+    through row-shifted descriptors); same results as the oracle and as the library's other kernels."""
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_conv(N, H_, W, C, K, R, S, 1, 0, 700 + N + H_ + C + K)
+    p.pad_h, p.pad_w = pad
+    want = H.conv_oracle(p)
+    assert want.shape == (N, H_ + 2 * pad[0] - R + 1, W + 2 * pad[1] - S + 1, K)
+    i8.set_path(0)
+    got = H.conv_gpu(p)
+    assert i8.last_path() == i8.PATH_CONV_SLAB, f"{p.name}: path {i8.last_path()}"
+    H.assert_same(got, want, p.name + " slab")
+    assert len(np.unique(want)) > 32, "degenerate output would prove nothing"
+    i8.set_path(3)
+    got = H.conv_gpu(p)
+    assert i8.last_path() != i8.PATH_CONV_SLAB
+    H.assert_same(got, want, p.name + " without the slab kernel")
+    assert i8.last_device_status() == 0
 
 
 def test_conv_1x1_equals_gemm_on_gpu():

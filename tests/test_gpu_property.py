@@ -55,8 +55,15 @@ def test_random_convs(N, H_, W, C32, K, R, stride, pad, seed, relu):
     want = H.conv_oracle(p)
     i8.set_path(0)
     got = H.conv_gpu(p)
-    assert i8.last_path() == i8.PATH_TENSOR
-    H.assert_same(got, want, f"{p.name} seed {seed}")
+    path = i8.last_path()
+    assert path in (i8.PATH_TENSOR, i8.PATH_CONV_SLAB)
+    H.assert_same(got, want, f"{p.name} seed {seed} path {path}")
+    if path == i8.PATH_CONV_SLAB:                       # stride-1 layers with few filters: also the implicit-GEMM kernel
+        i8.set_path(3)
+        got = H.conv_gpu(p)
+        assert i8.last_path() == i8.PATH_TENSOR
+        i8.set_path(0)
+        H.assert_same(got, want, f"{p.name} seed {seed} implicit GEMM")
 
 
 @settings(max_examples=15, deadline=None, suppress_health_check=list(HealthCheck))
