@@ -352,7 +352,7 @@ static int run_conv_slab(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_
     const int64_t reach = (int64_t)(BM + (R - 1) * Wp + S - 1) * cb;          // furthest byte any tap's 128 rows touch
     const int64_t stage_bytes = up1k(slab_tx > reach ? slab_tx : reach);
     const int64_t w_bytes = (int64_t)R * S * C * bn;                           // resident filter bank, zero rows up to bn
-    const int64_t fixed = up1k(w_bytes) + 9 * bn * 4 + (2 * SLAB_MAX_STAGES + 5) * 8 + 16;
+    const int64_t fixed = up1k(w_bytes) + 9 * bn * 4 + (2 * SLAB_MAX_STAGES + 2 * SLAB_ACC + 1) * 8 + 16;
     const int64_t budget = 227 * 1024 - 1024;
     int64_t stages = (budget - fixed) / stage_bytes;
     if (stages > SLAB_MAX_STAGES) stages = SLAB_MAX_STAGES;
@@ -386,7 +386,7 @@ static int run_conv_slab(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_
     p.y_vec_ok = aligned16(y) && Kf % 16 == 0;
     p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);
     p.dev_status = ctx->dev_status;
-    const size_t smem = (size_t)p.off_bar + (2 * SLAB_MAX_STAGES + 5) * 8 + 16 + 1024;
+    const size_t smem = (size_t)p.off_bar + (2 * SLAB_MAX_STAGES + 2 * SLAB_ACC + 1) * 8 + 16 + 1024;
     const int grid = p.num_tiles < ctx->sm_count ? p.num_tiles : ctx->sm_count;
     // 3 x 3 filters get the instance whose issue loop is unrolled over the nine taps
     void (*kern)(CUtensorMap, CUtensorMap, ConvSlabParams);

@@ -23,6 +23,7 @@ namespace i8 {
 constexpr int SLAB_MAX_STAGES = 8;
 constexpr int SLAB_THREADS = 32 * 3 + 32 * 8;     // producer, MMA issuer, 8 epilogue warps, second MMA issuer
 constexpr int SLAB_ISSUER2_WARP = 10;
+constexpr int SLAB_ACC = 4;                       // accumulators: the issuers may run this many tiles ahead of the read-out
 
 struct ConvSlabParams {
     int8_t* y;
@@ -65,7 +66,7 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     constexpr int EPI_THREADS = 256;
     constexpr int COLS_PER_GROUP = BN / 2;            // two warps share a lane quarter and split the columns
     static_assert(BN == 64 || BN == 128, "filter tiles of 64 or 128");
-    constexpr int TMEM_COLS = 2 * BN;
+    constexpr int TMEM_COLS = SLAB_ACC * BN;         // 256 or 512 columns
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -84,10 +85,10 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     const uint32_t bar_full = sbase + p.off_bar;
     const uint32_t bar_empty = bar_full + SLAB_MAX_STAGES * 8;
     const uint32_t bar_acc_full = bar_empty + SLAB_MAX_STAGES * 8;
-    const uint32_t bar_acc_empty = bar_acc_full + 2 * 8;
-    const uint32_t bar_w = bar_acc_empty + 2 * 8;
-    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + p.off_bar + (2 * SLAB_MAX_STAGES + 5) * 8);
-    volatile int* s_stop = reinterpret_cast<volatile int*>(smem + p.off_bar + (2 * SLAB_MAX_STAGES + 5) * 8 + 4);
+    const uint32_t bar_acc_empty = bar_acc_full + SLAB_ACC * 8;
+    const uint32_t bar_w = bar_acc_empty + SLAB_ACC * 8;
+    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + p.off_bar + (2 * SLAB_MAX_STAGES + 2 * SLAB_ACC + 1) * 8);
+    volatile int* s_stop = reinterpret_cast<volatile int*>(smem + p.off_bar + (2 * SLAB_MAX_STAGES + 2 * SLAB_ACC + 1) * 8 + 4);
 
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
     const int lane = threadIdx.x & 31;
@@ -99,7 +100,7 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
-        for (int b = 0; b < 2; b++) {
+        for (int b = 0; b < SLAB_ACC; b++) {
             mbar_init(bar_acc_full + 8 * b, 1);
             mbar_init(bar_acc_empty + 8 * b, EPI_THREADS);
         }
@@ -175,10 +176,10 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         __syncwarp();
     } else if (warp == 1 || warp == SLAB_ISSUER2_WARP) {
         // ------------------------------------------------------------------ MMA issuers
-        // Two warps issue: warp 1 the even tiles of this CTA's sequence (accumulator 0), the last warp the odd ones
-        // (accumulator 1).  A 128 x 64 x 32 instruction lasts ~50 cycles and the tensor core's queue is short, so one
-        // thread's barrier round trips between tiles would leave the tensor core idle; two independent streams into
-        // different accumulators fill each other's gaps.
+        // Two warps issue: warp 1 the even tiles of this CTA's sequence (even accumulators), the last warp the odd ones
+        // (odd accumulators).  A 128 x 64 x 32 instruction lasts ~50 cycles and the tensor core's queue is short, so
+        // one thread's barrier round trips between tiles would leave the tensor core idle; two independent streams
+        // into different accumulators fill each other's gaps.
         const int iss = warp == 1 ? 0 : 1;
         constexpr uint32_t idesc = make_idesc_i8(BM, BN, 0, 0);
         const uint64_t swz = p.cb == 128 ? SWZ_128B : (p.cb == 64 ? SWZ_64B : SWZ_32B);
@@ -203,7 +204,7 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                 tap_b[t] = b_base + (uint32_t)t * tap_units;
             }
         }
-        const int ab = iss;
+        int ab = iss;
         const int first = (int)blockIdx.x + iss * (int)gridDim.x;        // this issuer's first tile; it takes every second one
         int stage = 0;
         uint32_t phase = 0, acc_phase = 0;
@@ -252,7 +253,8 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             if (!ok) break;
             if (leader) tc_commit(bar_acc_full + 8 * ab);
             __syncwarp();
-            acc_phase ^= 1;
+            ab += 2;
+            if (ab >= SLAB_ACC) { ab -= SLAB_ACC; acc_phase ^= 1; }
             for (int c = 0; c < p.cblocks; c++)                          // the other issuer's tile in between
                 if (++stage == stages) { stage = 0; phase ^= 1; }
         }
@@ -322,8 +324,7 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             }
             tc_fence_before();
             mbar_arrive(bar_acc_empty + 8 * ab);
-            ab ^= 1;
-            if (ab == 0) acc_phase ^= 1;
+            if (++ab == SLAB_ACC) { ab = 0; acc_phase ^= 1; }
         }
     }
 
