@@ -42,6 +42,7 @@ static int g_pdl = 1;                            // programmatic dependent launc
 static int g_tc2 = 1;                            // two-SM GEMM kernel for large shapes (I8OPS_TC2=0 turns it off)
 static int g_conv_two_sm = -1;                   // CTA pairs for convolutions: -1 by rule, 0 never, 1 always (I8OPS_CONV2SM)
 static int g_force_bn = -1;                      // tuning override from the environment (I8OPS_FORCE_BN)
+static int g_sticky = 1;                         // column-sticky tile order for short-K problems (I8OPS_STICKY=0 turns it off)
 static int g_slab = 1;                           // slab-resident stride-1 convolution kernel (I8OPS_SLAB=0 turns it off)
 
 static thread_local int t_last_path = I8_PATH_NONE;
@@ -96,6 +97,8 @@ static int get_ctx(DeviceCtx** out) {
         if (c2) g_conv_two_sm = atoi(c2);
         const char* tc2 = getenv("I8OPS_TC2");
         if (tc2) g_tc2 = atoi(tc2);
+        const char* sticky = getenv("I8OPS_STICKY");
+        if (sticky) g_sticky = atoi(sticky);
         const char* slab = getenv("I8OPS_SLAB");
         if (slab) g_slab = atoi(slab);
         const char* pdl = getenv("I8OPS_PDL");
@@ -234,6 +237,20 @@ static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA
     p.sched.n_tiles = (N + bn - 1) / bn;
     p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
     p.sched.group_m = 16;                              // measured best of 2..32 on 8192^3 for the two-SM kernel
+    p.sched.sticky = 0; p.sched.col_base = 0; p.sched.col_rem = 0;
+    {
+        // Column-sticky order for short-K problems with several tiles per worker: rebuilding the epilogue constants for
+        // a new block column costs about as much as a short tile, so a worker keeps its column if that needs no more
+        // rounds than the raster order.
+        const int workers = two_sm ? ctx->sm_count / 2 : ctx->sm_count;
+        const int nt = p.sched.n_tiles, mt = p.sched.m_tiles;
+        if (g_sticky && nt > 1 && workers >= 2 * nt && p.sched.num_tiles > workers && kl.num_iters <= 16) {
+            const int base = workers / nt;
+            const int rounds_sticky = (mt + base - 1) / base;
+            const int rounds_raster = (p.sched.num_tiles + workers - 1) / workers;
+            if (rounds_sticky <= rounds_raster) { p.sched.sticky = 1; p.sched.col_base = base; p.sched.col_rem = workers % nt; }
+        }
+    }
     p.kl = kl;
     // resident B: one block column, and all of B's K blocks fit the ring's B region
     p.kl.b_resident = (p.sched.n_tiles == 1 && (int64_t)kl.num_kblocks * b_rows * kl.cb <= (int64_t)stages * b_rows * BK) ? 1 : 0;

@@ -51,9 +51,28 @@ __device__ __forceinline__ int fast_div(int n, int d, uint32_t inv) {
     return q;
 }
 
+// Two tile orders.  Grouped raster (sticky == 0): worker w takes tiles w, w + W, w + 2W, ... of a raster that walks
+// group_m block rows at a time through all block columns (L2 reuse for the large problems).  Column-sticky (sticky != 0,
+// chosen by the host for short-K problems with several tiles per worker): worker w owns block column w % n_tiles for the
+// whole kernel and walks its rows slot, slot + S, slot + 2S, ... (S = workers of that column), so the per-channel
+// epilogue constants are built once per CTA instead of once per tile.
 struct TileSched {
     int m_tiles, n_tiles, num_tiles, group_m;
-    __device__ __forceinline__ void map(int tile, int& m_blk, int& n_blk) const {
+    int sticky, col_base, col_rem;        // column-sticky order: every column has col_base workers, the first col_rem one more
+    // one past the last tile index of worker w (tiles advance by `step` = number of workers)
+    __device__ __forceinline__ int end_for(int w, int step) const {
+        if (!sticky) return num_tiles;
+        const int c = w % n_tiles, slot = w / n_tiles, S = col_base + (c < col_rem ? 1 : 0);
+        const int count = slot < m_tiles ? (m_tiles - slot + S - 1) / S : 0;
+        return w + count * step;
+    }
+    __device__ __forceinline__ void map(int tile, int w, int step, int& m_blk, int& n_blk) const {
+        if (sticky) {
+            const int it = (tile - w) / step;
+            n_blk = w % n_tiles;
+            m_blk = w / n_tiles + it * (col_base + (n_blk < col_rem ? 1 : 0));
+            return;
+        }
         if (n_tiles == 1) { m_blk = tile; n_blk = 0; return; }   // one block column: no divisions
         const int width = group_m * n_tiles;
         const int g = tile / width;
@@ -290,6 +309,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // persistent schedule: CTA (or CTA pair) w takes tiles w, w + W, w + 2W, ...
     const int first_tile = TWO_SM ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int tile_step = TWO_SM ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int tile_end = sched.end_for(first_tile, tile_step);
     // barriers of the even CTA, as seen from this CTA (its own in the one-SM kernel)
     const uint32_t full0 = TWO_SM ? map_to_cta(bar_full, 0) : bar_full;
     const uint32_t bres0 = TWO_SM ? map_to_cta(bar_bres, 0) : bar_bres;
@@ -306,7 +326,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         bool ok = true;
         const bool leader = elect_one();
         const bool bres = kl.b_resident != 0;
-        if (bres && pid == 0 && first_tile < sched.num_tiles && leader) {
+        if (bres && pid == 0 && first_tile < tile_end && leader) {
             // the paper's "keep B resident" step: the whole (small) B operand is fetched once per CTA into the
             // region the ring would otherwise use for B, and only A streams
             if (rank == 0) mbar_expect_tx(bar_bres, tx_mult * kl.num_kblocks * b_sub_bytes);
@@ -316,9 +336,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
         }
         const uint32_t stage_tx = a_sub_bytes + (bres ? 0u : b_sub_bytes);
-        for (int tile = first_tile; ok && tile < sched.num_tiles; tile += tile_step) {
+        for (int tile = first_tile; ok && tile < tile_end; tile += tile_step) {
             int m_blk, n_blk;
-            sched.map(tile, m_blk, n_blk);
+            sched.map(tile, first_tile, tile_step, m_blk, n_blk);
             const int row_a = m_blk * TILE_M + (int)rank * BM;          // this CTA's first A row (output row / pixel)
             const int row_b = n_blk * BN + (int)rank * B_ROWS;          // this CTA's first B row (output column)
             int w0 = 0, h0 = 0, img = 0;
@@ -371,7 +391,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (*s_stop && rank == 0) {
             // stopping early: let every copy this warp started land before the CTA retires (in a pair the even CTA's
             // barriers also count the odd CTA's copies, and the closing cluster barrier keeps the odd CTA alive meanwhile)
-            if (bres && pid == 0 && first_tile < sched.num_tiles && !mbar_wait_drain(bar_bres, 0, p.wait_limit_cycles))
+            if (bres && pid == 0 && first_tile < tile_end && !mbar_wait_drain(bar_bres, 0, p.wait_limit_cycles))
                 atomicCAS(p.dev_status, 0u, (unsigned)DEV_TIMEOUT_DRAIN);
             for (int s = 0; s < STAGES; s++)
                 if (issued & (1u << s))
@@ -405,8 +425,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const bool bres = kl.b_resident != 0;
         const uint32_t b_iter_units = (kl.nsub * b_sub_bytes) >> 4;   // resident B: descriptor units per ring slot's worth of K
         if (rank != 0) ok = false;                       // in a pair only the even CTA issues
-        if (ok && bres && first_tile < sched.num_tiles) ok = mbar_wait_warp(bar_bres, 0, env, DEV_TIMEOUT_MMA_FULL);
-        for (int tile = first_tile; ok && tile < sched.num_tiles; tile += tile_step) {
+        if (ok && bres && first_tile < tile_end) ok = mbar_wait_warp(bar_bres, 0, env, DEV_TIMEOUT_MMA_FULL);
+        for (int tile = first_tile; ok && tile < tile_end; tile += tile_step) {
             if (!mbar_wait_warp(bar_acc_empty + 8 * ab, acc_phase ^ 1, env, DEV_TIMEOUT_MMA_ACC)) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + ab * BN;
@@ -460,9 +480,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         long long rc[ONE_CHUNK ? 32 : 1];
         uint32_t acc_phase = 0;
         bool dead = false;
-        for (int tile = first_tile; tile < sched.num_tiles; tile += tile_step) {
+        for (int tile = first_tile; tile < tile_end; tile += tile_step) {
             int m_blk, n_blk;
-            sched.map(tile, m_blk, n_blk);
+            sched.map(tile, first_tile, tile_step, m_blk, n_blk);
             const int n0 = n_blk * BN;
             if (n_blk != cached_n_blk) {
                 // new block column: rebuild the per-channel constants (before waiting, so this overlaps the main loop)

@@ -200,6 +200,21 @@ def test_two_sm_kernel_shapes(M, N, K):
     _both_paths(p, two_sm=True)
 
 
+@pytest.mark.parametrize("M,N,K", [
+    (5000, 640, 256),      # 40 x 5 tiles of 128 x 128 over 148 CTAs: 29 or 30 workers per column, two rounds
+    (3136, 2048, 512),     # the 1x1 convolution of the ResNet-like mix as a GEMM: 25 x 16 tiles, 9 or 10 workers per column
+    (9001, 300, 64),       # ragged rows and columns, one K block
+    (4100, 1000, 1104),    # nine K blocks, last one partial
+    (20000, 520, 192),     # many rounds per worker
+])
+def test_column_sticky_tile_order(M, N, K):
+    """Short-K problems with several tiles per CTA: each CTA keeps one block column (the epilogue constants are built
+    once); every output tile must still be produced exactly once."""
+    p = inputs.make_gemm(M, N, K, 77 + M + N, per_channel=1, relu=0)
+    want = _both_paths(p)
+    H.not_degenerate(want)
+
+
 @pytest.mark.parametrize("M,N,K,pinned", [(300, 200, 112, False), (2048, 512, 256, True), (5000, 384, 160, True), (8192, 256, 128, False)])
 def test_host_buffer_variant(M, N, K, pinned):
     """gemm_i8_host: host buffers in, host buffer out (row chunks pipelined over three streams for M >= 2048)."""
