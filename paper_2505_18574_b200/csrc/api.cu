@@ -239,6 +239,14 @@ static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA
     p.sched.group_m = 16;                              // measured best of 2..32 on 8192^3 for the two-SM kernel
     p.sched.sticky = 0; p.sched.col_base = 0; p.sched.col_rem = 0;
     {
+        auto inv32 = [](int d) { return d <= 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)d); };
+        const int workers = two_sm ? ctx->sm_count / 2 : ctx->sm_count;
+        p.sched.inv_nt = inv32(p.sched.n_tiles);
+        p.sched.inv_width = inv32(p.sched.group_m * p.sched.n_tiles);
+        p.sched.inv_gm = inv32(p.sched.group_m);
+        p.sched.inv_step = inv32(p.sched.num_tiles < workers ? p.sched.num_tiles : workers);
+    }
+    {
         // Column-sticky order for short-K problems with several tiles per worker: rebuilding the epilogue constants for
         // a new block column costs about as much as a short tile, so a worker keeps its column if that needs no more
         // rounds than the raster order.

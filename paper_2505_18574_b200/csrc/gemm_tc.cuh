@@ -59,28 +59,32 @@ __device__ __forceinline__ int fast_div(int n, int d, uint32_t inv) {
 struct TileSched {
     int m_tiles, n_tiles, num_tiles, group_m;
     int sticky, col_base, col_rem;        // column-sticky order: every column has col_base workers, the first col_rem one more
+    // floor(2^32 / d) for the divisors below (0xffffffff for d == 1): a division costs a multiply and a fix-up instead
+    // of the ~150-cycle software routine, which matters between the microsecond tiles of the small problems
+    uint32_t inv_nt, inv_width, inv_gm, inv_step;     // n_tiles, group_m * n_tiles, group_m, number of workers
     // one past the last tile index of worker w (tiles advance by `step` = number of workers)
     __device__ __forceinline__ int end_for(int w, int step) const {
         if (!sticky) return num_tiles;
-        const int c = w % n_tiles, slot = w / n_tiles, S = col_base + (c < col_rem ? 1 : 0);
+        const int slot = fast_div(w, n_tiles, inv_nt), c = w - slot * n_tiles, S = col_base + (c < col_rem ? 1 : 0);
         const int count = slot < m_tiles ? (m_tiles - slot + S - 1) / S : 0;
         return w + count * step;
     }
     __device__ __forceinline__ void map(int tile, int w, int step, int& m_blk, int& n_blk) const {
         if (sticky) {
-            const int it = (tile - w) / step;
-            n_blk = w % n_tiles;
-            m_blk = w / n_tiles + it * (col_base + (n_blk < col_rem ? 1 : 0));
+            const int it = fast_div(tile - w, step, inv_step);
+            const int slot = fast_div(w, n_tiles, inv_nt);
+            n_blk = w - slot * n_tiles;
+            m_blk = slot + it * (col_base + (n_blk < col_rem ? 1 : 0));
             return;
         }
         if (n_tiles == 1) { m_blk = tile; n_blk = 0; return; }   // one block column: no divisions
         const int width = group_m * n_tiles;
-        const int g = tile / width;
+        const int g = fast_div(tile, width, inv_width);
         const int first_m = g * group_m;
         const int gsz = min(m_tiles - first_m, group_m);
         const int local = tile - g * width;
-        m_blk = first_m + local % gsz;
-        n_blk = local / gsz;
+        n_blk = gsz == group_m ? fast_div(local, group_m, inv_gm) : local / gsz;   // only the last, shorter group divides
+        m_blk = first_m + local - n_blk * gsz;
     }
 };
 
@@ -162,6 +166,20 @@ __device__ __forceinline__ void epilogue_chunk_fold(const int32_t (&v)[32], cons
         const longlong2 cb = *reinterpret_cast<const longlong2*>(s_c64 + c0 + 4 * j + 2);
         const uint32_t pk = pack_sat4(requant_fold(v[4 * j + 0], m2.x, ca.x), requant_fold(v[4 * j + 1], m2.y, ca.y),
                                       requant_fold(v[4 * j + 2], m2.z, cb.x), requant_fold(v[4 * j + 3], m2.w, cb.y));
+        out[j] = RELU ? relu_s8x4(pk) : pk;
+    }
+}
+// Folded form with the bias added explicitly: two words per channel from shared memory instead of three (a 16-byte
+// shared-memory broadcast costs four wavefronts, and eight epilogue warps each fetch every channel's constants).
+template <bool RELU>
+__device__ __forceinline__ void epilogue_chunk_fold_add(const int32_t (&v)[32], const int32_t* s_bias, const int32_t* s_m2, int c0,
+                                                        uint32_t (&out)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+        const int4 bi = *reinterpret_cast<const int4*>(s_bias + c0 + 4 * j);
+        const int4 m2 = *reinterpret_cast<const int4*>(s_m2 + c0 + 4 * j);
+        const uint32_t pk = pack_sat4(requant_fold(v[4 * j + 0] + bi.x, m2.x, 1ll << 31), requant_fold(v[4 * j + 1] + bi.y, m2.y, 1ll << 31),
+                                      requant_fold(v[4 * j + 2] + bi.z, m2.z, 1ll << 31), requant_fold(v[4 * j + 3] + bi.w, m2.w, 1ll << 31));
         out[j] = RELU ? relu_s8x4(pk) : pk;
     }
 }
@@ -543,8 +561,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                         if (p.relu) epilogue_chunk_fold_regs<true>(v, rm, rc, out);
                         else epilogue_chunk_fold_regs<false>(v, rm, rc, out);
                     } else {
-                        if (p.relu) epilogue_chunk_fold<true>(v, s_m2, s_c64, c0, out);
-                        else epilogue_chunk_fold<false>(v, s_m2, s_c64, c0, out);
+                        if (p.relu) epilogue_chunk_fold_add<true>(v, s_bias, s_m2, c0, out);
+                        else epilogue_chunk_fold_add<false>(v, s_bias, s_m2, c0, out);
                     }
                 } else if (shift32) {
                     // ReLU with a negative multiplier somewhere in the block column: ReLU must stay ahead of the scale
