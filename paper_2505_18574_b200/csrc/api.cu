@@ -245,6 +245,9 @@ static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA
         p.sched.inv_width = inv32(p.sched.group_m * p.sched.n_tiles);
         p.sched.inv_gm = inv32(p.sched.group_m);
         p.sched.inv_step = inv32(p.sched.num_tiles < workers ? p.sched.num_tiles : workers);
+        const int last = p.sched.m_tiles % p.sched.group_m;
+        p.sched.inv_last = inv32(last ? last : p.sched.group_m);
+        p.sched.inv_cb = 0xffffffffu; p.sched.inv_cb1 = 0xffffffffu;
     }
     {
         // Column-sticky order for short-K problems with several tiles per worker: rebuilding the epilogue constants for
@@ -256,7 +259,11 @@ static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA
             const int base = workers / nt;
             const int rounds_sticky = (mt + base - 1) / base;
             const int rounds_raster = (p.sched.num_tiles + workers - 1) / workers;
-            if (rounds_sticky <= rounds_raster) { p.sched.sticky = 1; p.sched.col_base = base; p.sched.col_rem = workers % nt; }
+            if (rounds_sticky <= rounds_raster) {
+                p.sched.sticky = 1; p.sched.col_base = base; p.sched.col_rem = workers % nt;
+                p.sched.inv_cb = base <= 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)base);
+                p.sched.inv_cb1 = (uint32_t)((1ull << 32) / (uint64_t)(base + 1));
+            }
         }
     }
     p.kl = kl;

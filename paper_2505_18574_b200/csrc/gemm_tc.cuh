@@ -62,11 +62,12 @@ struct TileSched {
     // floor(2^32 / d) for the divisors below (0xffffffff for d == 1): a division costs a multiply and a fix-up instead
     // of the ~150-cycle software routine, which matters between the microsecond tiles of the small problems
     uint32_t inv_nt, inv_width, inv_gm, inv_step;     // n_tiles, group_m * n_tiles, group_m, number of workers
+    uint32_t inv_last, inv_cb, inv_cb1;               // rows of the last (shorter) group, col_base, col_base + 1
     // one past the last tile index of worker w (tiles advance by `step` = number of workers)
     __device__ __forceinline__ int end_for(int w, int step) const {
         if (!sticky) return num_tiles;
         const int slot = fast_div(w, n_tiles, inv_nt), c = w - slot * n_tiles, S = col_base + (c < col_rem ? 1 : 0);
-        const int count = slot < m_tiles ? (m_tiles - slot + S - 1) / S : 0;
+        const int count = slot < m_tiles ? fast_div(m_tiles - slot + S - 1, S, c < col_rem ? inv_cb1 : inv_cb) : 0;
         return w + count * step;
     }
     __device__ __forceinline__ void map(int tile, int w, int step, int& m_blk, int& n_blk) const {
@@ -83,7 +84,7 @@ struct TileSched {
         const int first_m = g * group_m;
         const int gsz = min(m_tiles - first_m, group_m);
         const int local = tile - g * width;
-        n_blk = gsz == group_m ? fast_div(local, group_m, inv_gm) : local / gsz;   // only the last, shorter group divides
+        n_blk = gsz == group_m ? fast_div(local, group_m, inv_gm) : fast_div(local, gsz, inv_last);   // the last group may be shorter
         m_blk = first_m + local - n_blk * gsz;
     }
 };
@@ -341,7 +342,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int pid = warp == 0 ? 0 : 1;
         int stage = 0;
         uint32_t phase = 0, issued = 0, issued_phase = 0;
-        bool ok = true;
+        bool ok = true, first_pass = true;
         const bool leader = elect_one();
         const bool bres = kl.b_resident != 0;
         if (bres && pid == 0 && first_tile < tile_end && leader) {
@@ -377,10 +378,11 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     // the other producer's slot: only keep the tap / channel counters in step
                     for (int j = 0; j < nb; j++, kbi++)
                         if (CONV && ++c_idx == kl.cblocks) { c_idx = 0; if (++fs == kl.S) { fs = 0; ++fr; } }
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; first_pass = false; }
                     continue;
                 }
-                if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
+                // on the first pass over the ring every slot is free: nothing to wait for
+                if (!first_pass && !mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1, env, DEV_TIMEOUT_PRODUCER)) { ok = false; break; }
                 const uint32_t full = full0 + 8 * stage;
                 if (leader && rank == 0) mbar_expect_tx(bar_full + 8 * stage, tx_mult * nb * stage_tx);
                 for (int j = 0; j < nb; j++, kbi++) {
@@ -403,7 +405,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 }
                 issued |= 1u << stage;
                 issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
-                if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                if (++stage == STAGES) { stage = 0; phase ^= 1; first_pass = false; }
             }
         }
         if (*s_stop && rank == 0) {
