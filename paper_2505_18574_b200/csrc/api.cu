@@ -42,6 +42,7 @@ static int g_pdl = 1;                            // programmatic dependent launc
 static int g_tc2 = 1;                            // two-SM GEMM kernel for large shapes (I8OPS_TC2=0 turns it off)
 static int g_conv_two_sm = -1;                   // CTA pairs for convolutions: -1 by rule, 0 never, 1 always (I8OPS_CONV2SM)
 static int g_force_bn = -1;                      // tuning override from the environment (I8OPS_FORCE_BN)
+static int g_tma_store = 1;                      // read-out of the wide tiles through TMA stores (I8OPS_TMA_STORE=0 turns it off)
 static int g_sticky = 1;                         // column-sticky tile order for short-K problems (I8OPS_STICKY=0 turns it off)
 static int g_slab = 1;                           // slab-resident stride-1 convolution kernel (I8OPS_SLAB=0 turns it off)
 
@@ -97,6 +98,8 @@ static int get_ctx(DeviceCtx** out) {
         if (c2) g_conv_two_sm = atoi(c2);
         const char* tc2 = getenv("I8OPS_TC2");
         if (tc2) g_tc2 = atoi(tc2);
+        const char* tst = getenv("I8OPS_TMA_STORE");
+        if (tst) g_tma_store = atoi(tst);
         const char* sticky = getenv("I8OPS_STICKY");
         if (sticky) g_sticky = atoi(sticky);
         const char* slab = getenv("I8OPS_SLAB");
@@ -160,8 +163,8 @@ static CUtensorMapSwizzle swizzle_for(int cb) {
 }
 
 template <int BN, int STAGES, bool CONV, int EPI_WARPS, int NPROD, bool TWO_SM>
-static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUtensorMap& tmB, GemmTcParams& p,
-                     cudaStream_t st) {
+static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                     GemmTcParams& p, cudaStream_t st) {
     using L = TcSmem<BN, STAGES, TWO_SM>;
     auto kern = gemm_i8_tc_kernel<BN, STAGES, CONV, EPI_WARPS, NPROD, TWO_SM>;
     if (!ctx->attr_set[slot]) {
@@ -173,7 +176,7 @@ static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUt
     // short kernels gain from overlapping their launch with the predecessor's tail; long ones do not need it
     const bool overlap = !TWO_SM && 2.0 * p.M * p.N * p.K < 4e10;
     CUDA_TRY(launch_kernel(kern, overlap, TWO_SM ? 2 : 1, TWO_SM ? 2 * used : used, 32 * (1 + NPROD) + 32 * EPI_WARPS, L::DYN_BYTES,
-                           st, tmA, tmB, p));
+                           st, tmA, tmB, tmC, p));
     return I8_OK;
 }
 
@@ -233,6 +236,17 @@ static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA
     p.per_channel = per_channel; p.relu = relu; p.M = M; p.N = N; p.K = K;
     p.c_vec_ok = raw.D ? (aligned16(raw.D) && raw.ldd % 4 == 0) : (aligned16(C) && (ldc % 16 == 0));
     p.D = raw.D; p.ldd = raw.ldd; p.raw = raw.D ? 1 : 0; p.accumulate = raw.accumulate;
+    // wide tiles hand their int8 output to the TMA engine as 32-row x 64-byte boxes (needs a 16-byte aligned C)
+    CUtensorMap tmC = tmB;
+    p.tma_store = 0;
+    if (g_tma_store && !raw.D && bn >= 128 && p.c_vec_ok) {
+        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)M};
+        const uint64_t str[1] = {(uint64_t)ldc};
+        const uint32_t box[2] = {64, 32};
+        int rc = make_tmap(&tmC, C, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_64B);
+        if (rc) return rc;
+        p.tma_store = 1;
+    }
     p.sched.m_tiles = (M + tile_m - 1) / tile_m;
     p.sched.n_tiles = (N + bn - 1) / bn;
     p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
@@ -274,24 +288,24 @@ static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA
     if (two_sm) {
         if (conv) {
             switch (bn) {
-                case 256: return launch_tc<256, 6, true, 8, 2, true>(ctx, 8, tmA, tmB, p, st);
-                case 128: return launch_tc<128, 8, true, 8, 2, true>(ctx, 9, tmA, tmB, p, st);
-                default:  return launch_tc<64, 8, true, 8, 2, true>(ctx, 10, tmA, tmB, p, st);
+                case 256: return launch_tc<256, 6, true, 8, 2, true>(ctx, 8, tmA, tmB, tmC, p, st);
+                case 128: return launch_tc<128, 8, true, 8, 2, true>(ctx, 9, tmA, tmB, tmC, p, st);
+                default:  return launch_tc<64, 8, true, 8, 2, true>(ctx, 10, tmA, tmB, tmC, p, st);
             }
         }
-        return launch_tc<256, 6, false, 8, 1, true>(ctx, 7, tmA, tmB, p, st);
+        return launch_tc<256, 6, false, 8, 1, true>(ctx, 7, tmA, tmB, tmC, p, st);
     }
     if (conv) {
         switch (bn) {
-            case 256: return launch_tc<256, 4, true, 8, 2, false>(ctx, 3, tmA, tmB, p, st);
-            case 128: return launch_tc<128, 6, true, 8, 2, false>(ctx, 4, tmA, tmB, p, st);
-            default:  return launch_tc<64, 8, true, 8, 2, false>(ctx, 5, tmA, tmB, p, st);
+            case 256: return launch_tc<256, 4, true, 8, 2, false>(ctx, 3, tmA, tmB, tmC, p, st);
+            case 128: return launch_tc<128, 6, true, 8, 2, false>(ctx, 4, tmA, tmB, tmC, p, st);
+            default:  return launch_tc<64, 8, true, 8, 2, false>(ctx, 5, tmA, tmB, tmC, p, st);
         }
     }
     switch (bn) {
-        case 256: return launch_tc<256, 4, false, 8, 1, false>(ctx, 0, tmA, tmB, p, st);
-        case 128: return launch_tc<128, 6, false, 8, 1, false>(ctx, 1, tmA, tmB, p, st);
-        default:  return launch_tc<64, 8, false, 8, 1, false>(ctx, 2, tmA, tmB, p, st);
+        case 256: return launch_tc<256, 4, false, 8, 1, false>(ctx, 0, tmA, tmB, tmC, p, st);
+        case 128: return launch_tc<128, 6, false, 8, 1, false>(ctx, 1, tmA, tmB, tmC, p, st);
+        default:  return launch_tc<64, 8, false, 8, 1, false>(ctx, 2, tmA, tmB, tmC, p, st);
     }
 }
 

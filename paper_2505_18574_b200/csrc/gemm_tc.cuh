@@ -98,6 +98,7 @@ struct GemmTcParams {
     int per_channel, relu;
     int M, N, K;
     int c_vec_ok;               // C (or D) and its leading dimension are 16-byte aligned: full chunks go out as 16-byte stores
+    int tma_store;              // wide tiles: int8 output leaves through shared memory and TMA stores (tmC is valid)
     int32_t* D;                 // raw read-out: the int32 accumulators themselves, no bias / activation / scale
     int64_t ldd;
     int raw, accumulate;        // raw != 0 selects D; accumulate != 0 adds to what D already holds
@@ -117,7 +118,11 @@ struct TcSmem {
     static constexpr int OFF_CONST = OFF_B + STAGES * B_BYTES;       // 7 int32[BN] arrays and one int64[BN] array of per-channel constants
     static constexpr int OFF_BAR = OFF_CONST + 9 * BN * 4;           // full[S], empty[S], acc_full[2], acc_empty[2], b_resident
     static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 5) * 8;  // tensor-memory base, stop flag
-    static constexpr int TOTAL = OFF_MISC + 16;
+    // read-out staging of the wide tiles: every epilogue warp collects 32 rows x 64 output bytes (64-byte swizzle) and one
+    // lane hands them to the TMA engine: the 32 scattered row segments cost the load/store pipe nothing
+    static constexpr int STAGE_WARP_BYTES = 32 * 64;
+    static constexpr int OFF_STAGE = (OFF_MISC + 16 + 1023) / 1024 * 1024;
+    static constexpr int TOTAL = BN >= 128 ? OFF_STAGE + 8 * STAGE_WARP_BYTES : OFF_MISC + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;                   // slack to align the base to 1024 bytes
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // BN in {64,128,256}: a power of two
 };
@@ -227,7 +232,8 @@ __device__ __forceinline__ void store_raw_chunk(int32_t* drow, int n, int N, boo
 
 template <int BN, int STAGES, bool CONV, int EPI_WARPS, int NPROD, bool TWO_SM>
 __global__ void __launch_bounds__(32 * (1 + NPROD) + 32 * EPI_WARPS, 1)
-gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmTcParams p) {
+gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmC, const GemmTcParams p) {
     using L = TcSmem<BN, STAGES, TWO_SM>;
     constexpr int EPI_THREADS = 32 * EPI_WARPS;
     constexpr int TILE_M = TWO_SM ? 2 * BM : BM;       // rows of one output tile (a CTA pair shares a 256-row tile)
@@ -543,6 +549,10 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const int row = m_blk * TILE_M + (int)rank * BM + quarter * 32 + lane;
             int8_t* crow = p.C + (int64_t)row * p.ldc;
             const uint32_t t0 = tmem_base + ab * BN + ((uint32_t)(quarter * 32) << 16);
+            // staging buffer of this warp: row r holds four 16-byte units, unit u at position u ^ ((r >> 1) & 3) (the
+            // 64-byte TMA swizzle, which also keeps the row-wise 16-byte writes free of bank conflicts)
+            const uint32_t stage_w = sbase + L::OFF_STAGE + (warp - 2) * L::STAGE_WARP_BYTES;
+            const bool staged = !ONE_CHUNK && p.tma_store != 0;
 #pragma unroll 1
             for (int ch = 0; ch < COLS_PER_GROUP / 32; ch++) {
                 const int c0 = cgroup * COLS_PER_GROUP + ch * 32;
@@ -573,6 +583,32 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 } else {
                     epilogue_chunk(v, s_bias, s_lo, s_hi, s_mult, s_shift, s_rnd, c0, out);
                 }
+                if constexpr (!ONE_CHUNK) {
+                    if (staged) {
+                        if ((ch & 1) == 0) {
+                            // the previous pair's copy must have read the buffer before it is refilled
+                            if (lane == 0) tma_store_wait_read();
+                            __syncwarp();
+                        }
+                        const uint32_t srow = stage_w + lane * 64;
+                        const uint32_t sw = (lane >> 1) & 3, u0 = 2 * (ch & 1);
+                        st_shared_v4(srow + ((u0 ^ sw) << 4), out[0], out[1], out[2], out[3]);
+                        st_shared_v4(srow + (((u0 + 1) ^ sw) << 4), out[4], out[5], out[6], out[7]);
+                        // a pair is complete after its second chunk, or when the block column ends after the first
+                        if ((ch & 1) || n + 32 >= p.N) {
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            // rows beyond M and columns beyond N are clipped by the copy engine (stale bytes of an
+                            // unwritten second half only ever fall there)
+                            const int y0 = m_blk * TILE_M + (int)rank * BM + quarter * 32;
+                            if (lane == 0 && y0 < p.M) {
+                                tma_store_2d(&tmC, stage_w, n - 32 * (ch & 1), y0);
+                                tma_store_commit();
+                            }
+                        }
+                        continue;
+                    }
+                }
                 if (row < p.M) store_row_chunk(crow, n, p.N, p.c_vec_ok != 0, out);
             }
             tc_fence_before();
@@ -588,6 +624,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
     }
 
+    if (warp >= 2 && warp < 2 + EPI_WARPS && lane == 0) tma_store_wait_all();   // this lane's output copies are complete
     tc_fence_before();
     if (TWO_SM) {
         cluster_sync_all();        // neither CTA leaves or frees tensor memory while the other still works
