@@ -236,10 +236,12 @@ static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA
     p.per_channel = per_channel; p.relu = relu; p.M = M; p.N = N; p.K = K;
     p.c_vec_ok = raw.D ? (aligned16(raw.D) && raw.ldd % 4 == 0) : (aligned16(C) && (ldc % 16 == 0));
     p.D = raw.D; p.ldd = raw.ldd; p.raw = raw.D ? 1 : 0; p.accumulate = raw.accumulate;
-    // wide tiles hand their int8 output to the TMA engine as 32-row x 64-byte boxes (needs a 16-byte aligned C)
+    // wide tiles hand their int8 output to the TMA engine as 32-row x 64-byte boxes; needs a 16-byte aligned C and an N
+    // that is a multiple of 16: the copy engine clips a box at the tensor's edge in 16-byte units, so with a ragged N
+    // it would write up to 15 bytes past the last column
     CUtensorMap tmC = tmB;
     p.tma_store = 0;
-    if (g_tma_store && !raw.D && bn >= 128 && p.c_vec_ok) {
+    if (g_tma_store && !raw.D && bn >= 128 && p.c_vec_ok && N % 16 == 0) {
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)M};
         const uint64_t str[1] = {(uint64_t)ldc};
         const uint32_t box[2] = {64, 32};

@@ -191,7 +191,8 @@ __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorM
         : "memory");
 }
 
-// Tiled store from shared memory to global memory (the box is clipped at the tensor's extent; the innermost coordinate
+// Tiled store from shared memory to global memory (the box is clipped at the tensor's extent, in 16-byte units along the
+// innermost dimension: keep that extent a multiple of 16 bytes; the innermost coordinate
 // times the element size must be a multiple of 16 bytes and no coordinate may be negative).  The issuing thread groups
 // its stores with commit and waits on its own groups: `.read` = the shared-memory source may be overwritten,
 // without = the writes are complete.  Shared-memory writes made by ordinary stores must be fenced into the async

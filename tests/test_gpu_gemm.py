@@ -215,6 +215,20 @@ def test_column_sticky_tile_order(M, N, K):
     H.not_degenerate(want)
 
 
+@pytest.mark.parametrize("M,N,K,ldc_pad", [(1, 13, 16, 3), (130, 200, 64, 8), (257, 328, 128, 0), (300, 135, 48, 9), (64, 1000, 32, 24),
+                                           (513, 272, 256, 16), (100, 16, 16, 0)])
+def test_wide_tiles_never_write_outside_c(M, N, K, ldc_pad):
+    """The two-SM kernel (256-wide tiles, read-out through TMA stores where N is a multiple of 16) with ragged N, ragged M and a
+    padded leading dimension: the harness checks the padding columns and the guard bytes around C."""
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_gemm(M, N, K, 5 + M + N, per_channel=1, relu=0, ldc_pad=ldc_pad, shift_lo=10, shift_hi=16)
+    want = H.gemm_oracle(p)
+    for mode in (2, 0):
+        i8.set_path(mode)
+        H.assert_same(H.gemm_gpu(p), want, f"{p.name} mode {mode}")
+    i8.set_path(0)
+
+
 @pytest.mark.parametrize("M,N,K,pinned", [(300, 200, 112, False), (2048, 512, 256, True), (5000, 384, 160, True), (8192, 256, 128, False)])
 def test_host_buffer_variant(M, N, K, pinned):
     """gemm_i8_host: host buffers in, host buffer out (row chunks pipelined over three streams for M >= 2048)."""
