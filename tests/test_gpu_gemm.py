@@ -229,6 +229,24 @@ def test_wide_tiles_never_write_outside_c(M, N, K, ldc_pad):
     i8.set_path(0)
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_seeded_random_shapes_all_tile_orders(seed):
+    """Medium-sized random shapes (several tiles per CTA, ragged edges, padded C) on the automatic path and on the forced
+    two-SM path: exercises the raster and column-sticky tile orders, the TMA-store and direct read-outs and their edges."""
+    import paper_2505_18574_b200 as i8
+    rng = np.random.default_rng(1000 + seed)
+    M = int(rng.integers(1, 6000)); N = int(rng.choice([16, 48, 64, 100, 128, 200, 256, 384, 520, 777, 1024, 1500]))
+    K = 16 * int(rng.integers(1, 40))
+    p = inputs.make_gemm(M, N, K, 2000 + seed, per_channel=int(rng.integers(0, 2)), relu=int(rng.integers(0, 2)),
+                         ldc_pad=int(rng.choice([0, 0, 16, 5])), shift_lo=10, shift_hi=18)
+    want = H.gemm_oracle(p)
+    for mode in (0, 2):
+        i8.set_path(mode)
+        H.assert_same(H.gemm_gpu(p), want, f"{p.name} seed {seed} mode {mode}")
+    i8.set_path(0)
+    assert i8.last_device_status() == 0
+
+
 @pytest.mark.parametrize("M,N,K,pinned", [(300, 200, 112, False), (2048, 512, 256, True), (5000, 384, 160, True), (8192, 256, 128, False)])
 def test_host_buffer_variant(M, N, K, pinned):
     """gemm_i8_host: host buffers in, host buffer out (row chunks pipelined over three streams for M >= 2048)."""
