@@ -135,6 +135,33 @@ def test_conv_slab_kernel(N, H_, W, C, K, R, S, pad):
     assert i8.last_device_status() == 0
 
 
+@pytest.mark.parametrize("seed", range(16))
+def test_seeded_random_stride1_convs(seed):
+    """Random stride-1 layers up to the slab kernel's limits (raster width 128, 128 filters, filter bank in shared memory):
+    whichever kernel the dispatcher picks must agree with the oracle, and so must the implicit-GEMM / generic choice."""
+    import paper_2505_18574_b200 as i8
+    rng = np.random.default_rng(4000 + seed)
+    R = int(rng.choice([1, 3, 5])); S = int(rng.choice([1, 3, 5]))
+    ph = int(rng.integers(0, R // 2 + 1)); pw = int(rng.integers(0, S // 2 + 1))
+    W = int(rng.choice([S, 7, 14, 28, 56, 100, 124, 126, 128 - 2 * pw, 130]))
+    H_ = int(rng.integers(R, 30)); N = int(rng.integers(1, 5))
+    C = int(rng.choice([32, 64, 96, 128])); K = int(rng.choice([1, 8, 40, 64, 65, 100, 128, 136]))
+    if R == 1 and S == 1:
+        ph = pw = 1                                       # keep it off the 1x1 -> GEMM shortcut
+    p = inputs.make_conv(N, H_, W, C, K, R, S, 1, 0, 4100 + seed, relu=int(rng.integers(0, 2)))
+    p.pad_h, p.pad_w = ph, pw
+    want = H.conv_oracle(p)
+    paths = []
+    for mode in (0, 3):
+        i8.set_path(mode)
+        got = H.conv_gpu(p)
+        paths.append(i8.last_path())
+        H.assert_same(got, want, f"{p.name} pad ({ph},{pw}) seed {seed} mode {mode} path {paths[-1]}")
+    i8.set_path(0)
+    assert paths[1] != i8.PATH_CONV_SLAB
+    assert i8.last_device_status() == 0
+
+
 def test_conv_1x1_equals_gemm_on_gpu():
     p = inputs.make_conv(3, 7, 7, 128, 256, 1, 1, 1, 0, 8)
     y = H.conv_gpu(p)
