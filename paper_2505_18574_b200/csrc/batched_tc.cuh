@@ -23,7 +23,7 @@ namespace i8 {
 
 constexpr int PAIR_UMMA_K = 32;                     // K per tcgen05.mma for 8-bit operands
 constexpr int PAIR_ACC = 4;                         // accumulators = epilogue groups
-constexpr int PAIR_STAGES = 8;                      // ring slots
+constexpr int PAIR_STAGES = 4;                      // ring slots (measured: 3 to 5 are equally fast, 8 and 12 slower)
 constexpr int PAIR_TILE_BYTES = 2 * 64 * 64;        // one operand of a pair
 constexpr int PAIR_THREADS = 64 + 128 * PAIR_ACC;
 
