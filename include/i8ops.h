@@ -137,6 +137,10 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y,
  * back and synchronises `stream` before returning.  Problems with 2048 rows or more are cut into row chunks whose
  * copy-in, kernel and copy-out overlap on three streams (two of them internal).  They also check every shift (I8_ERR_RANGE).
  * Tight layouts only: A row-major [M][K], B column-major (K contiguous, [N][K]), C row-major [M][N].
+ * The workspace, the internal streams and their events belong to the device, not to the call: calls on one device are
+ * serialised by a lock inside the library (a second host thread waits until the first call has returned), so
+ * concurrent callers are safe but gain nothing.  If a CUDA call fails part-way, everything already queued is allowed
+ * to finish before the error is returned; C is then unspecified.
  */
 int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C,
                  const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
@@ -194,20 +198,58 @@ int mpc_forward_f32(const float* Adyn, const float* Bdyn, const float* Kinf, con
  * for one GEMM is replayed on GEMMs of the same aspect class: square, column-dominant, row-dominant). */
 typedef struct {
     int shape_class;     /* 0 square (neither side 8x the other), 1 column-dominant (M >= 8N), 2 row-dominant (N >= 8M) */
-    int tile_m, tile_n;  /* output tile: 128 x {64, 128, 256} */
+    int tile_m, tile_n;  /* output tile: 128 (one CTA) or 256 (a CTA pair) x {64, 128, 256} */
     int stages;          /* ring slots of 128 bytes of K */
-    int m_tiles, n_tiles, waves;
+    int cta_group;       /* 1: one CTA per tile; 2: a cluster of two CTAs per tile (tcgen05.mma.cta_group::2) */
+    int raster_group;    /* block rows walked through all block columns before moving on (L2 reuse) */
+    int sticky;          /* 1: every worker keeps one block column for the whole kernel */
+    int m_tiles, n_tiles;
+    int workers;         /* CTAs (cta_group 1) or CTA pairs (cta_group 2) launched */
+    int waves;           /* ceil(tiles / workers) */
     int b_resident;      /* B fetched once per CTA and kept in shared memory */
     int epilogue_warps;
 } i8_plan;
 
-/* Fills *out with the plan gemm_i8 would use for (M, N, K) on a device with sm_count SMs.  Host only; no CUDA call.
+/* Fills *out with the plan gemm_i8 would launch for K-contiguous operands of shape (M, N, K) on a device with sm_count
+ * SMs: the launch code and this query call the same planning function.  Host only; no CUDA call.
  * Errors: I8_ERR_NULL, I8_ERR_SHAPE (a non-positive argument). */
 int i8ops_plan_gemm(int M, int N, int K, int sm_count, i8_plan* out);
 
-/* Records tile_n (64, 128 or 256; 0 forgets) as the tile width of every later shape of class shape_class, instead of
- * the built-in cost model (a width wider than the problem is ignored).  Errors: I8_ERR_RANGE. */
+/* The plan of the most recent launch of the large-tile tensor kernel made by this thread (GEMM or convolution). */
+int i8ops_last_plan(i8_plan* out);
+
+/* Records a schedule for every later GEMM of class shape_class (the paper's reuse of one shape's schedule on the other
+ * shapes of its class), replacing the built-in choice for the fields that are set:
+ *   base_m, base_n, base_k   the shape the schedule was found on: the entry then applies to shapes whose M, N and K each
+ *                            lie within a factor of four of it; all three 0: the entry applies to the whole class
+ *   tile_n        64, 128 or 256; 0 = cost model (a width much wider than the problem is ignored)
+ *   cta_group     1 or 2; 0 = measured crossover rule (2 implies 256-wide tiles)
+ *   raster_group  1..64; 0 = default (16)
+ *   sticky        1 = column-sticky order where it is legal, 0 = never, -1 = rule
+ * All fields at "no choice" forgets the entry.  The library starts with two entries, seeded from its tuned plans for
+ * 8192^3 (square) and 262144 x 64 x 256 (column-dominant).  Not thread-safe against concurrent launches.
+ * Errors: I8_ERR_RANGE. */
+int i8ops_set_class_plan(int shape_class, int base_m, int base_n, int base_k, int tile_n, int cta_group, int raster_group,
+                         int sticky);
+
+/* Shorthand: record only a tile width for the whole class (tile_n == 0 forgets the class entry). */
 int i8ops_set_class_tile(int shape_class, int tile_n);
+
+/* Tensor maps are cached per host thread, keyed on base address and geometry.  Reports this thread's cache hits and
+ * misses so far (for tests and tuning).  Errors: I8_ERR_NULL. */
+int i8ops_tmap_cache_stats(uint64_t* hits, uint64_t* misses);
+
+/* Measures the issue rate of the tensor-core instruction every int8 kernel here is built on (no counterpart in the
+ * paper; it gives the roofline its measured int8 denominator).  `ctas` CTAs, one per SM, each issue `reps`
+ * tcgen05.mma kind::i8 instructions of 128 x tile_n x 32 on operands that already sit in shared memory and wait for
+ * the last to finish.  Asynchronous on `stream`.
+ *   out   device, uint64 [ctas][4], written by the kernel: SM cycles spent issuing; SM cycles until the last
+ *         instruction completed; nanoseconds (global timer) until then; the SM's id.  A CTA whose bounded wait expired
+ *         writes 0 for the second and third value.
+ *   Peak of the chip = ctas * reps * 2 * 128 * tile_n * 32 operations / the largest of the nanosecond figures.
+ * Errors: I8_ERR_NULL, I8_ERR_RANGE (tile_n not a multiple of 16 in 16..256, reps not a multiple of 64 in 64..2^24,
+ * ctas outside 1..SM count), I8_ERR_CUDA. */
+int i8ops_probe_mma_rate(int tile_n, int reps, int ctas, unsigned long long* out, void* stream);
 
 /* Self-test of the failure path (no counterpart in the paper): launches one small CTA that waits, for at most
  * `limit_ms` (1..1000) milliseconds, on a barrier that nothing signals.  The kernel returns by itself and the next

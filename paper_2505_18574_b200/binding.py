@@ -35,6 +35,10 @@ SIGNATURES = {
     "i8ops_selftest_bounded_wait": (_int, [_int, _vp]),
     "i8ops_plan_gemm": (_int, [_int, _int, _int, _int, _vp]),
     "i8ops_set_class_tile": (_int, [_int, _int]),
+    "i8ops_set_class_plan": (_int, [_int] * 8),
+    "i8ops_last_plan": (_int, [_vp]),
+    "i8ops_tmap_cache_stats": (_int, [_vp, _vp]),
+    "i8ops_probe_mma_rate": (_int, [_int, _int, _int, _vp, _vp]),
     "i8ops_last_cuda_error": (_int, []),
     "i8ops_last_path": (_int, []),
     "i8ops_set_path": (_int, [_int]),
@@ -87,15 +91,18 @@ def _ptr(t) -> Optional[int]:
     return None if t is None else t.data_ptr()
 
 
-def gemm_i8(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:
-    """C = epilogue(A . B).  A: (M, K) int8 view, B: (K, N) int8 view (pass ``Bt.t()`` for a column-major B
-    stored as (N, K)), C: (M, N) int8 with unit column stride; bias int32 [N] or None; mult/shift int32 [1] or [N]."""
+def _gemm_i8_args(A, B, C, bias, mult, shift, per_channel, relu, stream=None):
     M, K = A.shape
     K2, N = B.shape
     assert K == K2 and tuple(C.shape) == (M, N) and (C.stride(1) == 1 or N <= 1)
-    st = lib().gemm_i8(_ptr(A), A.stride(0), A.stride(1), _ptr(B), B.stride(0), B.stride(1), _ptr(C), C.stride(0),
-                       _ptr(bias), _ptr(mult), _ptr(shift), int(per_channel), M, N, K, int(relu), _stream_ptr(stream))
-    _check(st, "gemm_i8")
+    return (_ptr(A), A.stride(0), A.stride(1), _ptr(B), B.stride(0), B.stride(1), _ptr(C), C.stride(0),
+            _ptr(bias), _ptr(mult), _ptr(shift), int(per_channel), M, N, K, int(relu), _stream_ptr(stream))
+
+
+def gemm_i8(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:
+    """C = epilogue(A . B).  A: (M, K) int8 view, B: (K, N) int8 view (pass ``Bt.t()`` for a column-major B
+    stored as (N, K)), C: (M, N) int8 with unit column stride; bias int32 [N] or None; mult/shift int32 [1] or [N]."""
+    _check(lib().gemm_i8(*_gemm_i8_args(A, B, C, bias, mult, shift, per_channel, relu, stream)), "gemm_i8")
 
 
 def gemm_i8_raw(A, B, D, accumulate: bool = False, stream=None) -> None:
@@ -108,29 +115,66 @@ def gemm_i8_raw(A, B, D, accumulate: bool = False, stream=None) -> None:
     _check(st, "gemm_i8_raw")
 
 
-def batched_gemm_i8(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:
-    """A: (batch, M, K), B: (batch, K, N), C: (batch, M, N) int8 views; bias int32 (batch, N), (N,) or None."""
+def _batched_gemm_i8_args(A, B, C, bias, mult, shift, per_channel, relu, stream=None):
     batch, M, K = A.shape
     _, K2, N = B.shape
     assert K == K2 and tuple(C.shape) == (batch, M, N) and (C.stride(2) == 1 or N <= 1)
     bias_bs = 0
     if bias is not None and bias.dim() == 2:
         bias_bs = bias.stride(0)
-    st = lib().batched_gemm_i8(_ptr(A), A.stride(1), A.stride(2), A.stride(0), _ptr(B), B.stride(1), B.stride(2),
-                               B.stride(0), _ptr(C), C.stride(1), C.stride(0), _ptr(bias), bias_bs, _ptr(mult),
-                               _ptr(shift), int(per_channel), batch, M, N, K, int(relu), _stream_ptr(stream))
-    _check(st, "batched_gemm_i8")
+    return (_ptr(A), A.stride(1), A.stride(2), A.stride(0), _ptr(B), B.stride(1), B.stride(2), B.stride(0), _ptr(C),
+            C.stride(1), C.stride(0), _ptr(bias), bias_bs, _ptr(mult), _ptr(shift), int(per_channel), batch, M, N, K,
+            int(relu), _stream_ptr(stream))
+
+
+def batched_gemm_i8(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:
+    """A: (batch, M, K), B: (batch, K, N), C: (batch, M, N) int8 views; bias int32 (batch, N), (N,) or None."""
+    _check(lib().batched_gemm_i8(*_batched_gemm_i8_args(A, B, C, bias, mult, shift, per_channel, relu, stream)),
+           "batched_gemm_i8")
+
+
+def _conv2d_i8_args(x, w, y, bias, mult, shift, per_channel, relu, stride=(1, 1), pad=(0, 0), stream=None):
+    N, H, W, C = x.shape
+    K, R, S, C2 = w.shape
+    assert C == C2 and x.is_contiguous() and w.is_contiguous() and y.is_contiguous()
+    return (_ptr(x), _ptr(w), _ptr(y), _ptr(bias), _ptr(mult), _ptr(shift), int(per_channel), N, H, W, C, K, R, S,
+            int(stride[0]), int(stride[1]), int(pad[0]), int(pad[1]), int(relu), _stream_ptr(stream))
 
 
 def conv2d_i8(x, w, y, bias, mult, shift, per_channel: int, relu: int, stride=(1, 1), pad=(0, 0), stream=None) -> None:
     """x: (N, H, W, C), w: (K, R, S, C), y: (N, P, Q, K), all dense int8."""
-    N, H, W, C = x.shape
-    K, R, S, C2 = w.shape
-    assert C == C2 and x.is_contiguous() and w.is_contiguous() and y.is_contiguous()
-    st = lib().conv2d_i8(_ptr(x), _ptr(w), _ptr(y), _ptr(bias), _ptr(mult), _ptr(shift), int(per_channel),
-                         N, H, W, C, K, R, S, int(stride[0]), int(stride[1]), int(pad[0]), int(pad[1]), int(relu),
-                         _stream_ptr(stream))
-    _check(st, "conv2d_i8")
+    _check(lib().conv2d_i8(*_conv2d_i8_args(x, w, y, bias, mult, shift, per_channel, relu, stride, pad, stream)), "conv2d_i8")
+
+
+class Prepared:
+    """One call into the C ABI with its arguments marshalled ahead of time: ``prepare("gemm_i8", A, B.t(), C, ...)``
+    reads pointers, extents and strides from the tensors once; calling the object then only crosses the boundary (what a
+    C caller's loop does).  The tensors must stay alive and unmoved, and the stream is the one current at preparation."""
+
+    _ARGS = {"gemm_i8": _gemm_i8_args, "batched_gemm_i8": _batched_gemm_i8_args, "conv2d_i8": _conv2d_i8_args}
+
+    def __init__(self, name: str, *tensors, **kw):
+        self.name = name
+        self._fn = getattr(lib(), name)
+        raw = self._ARGS[name](*tensors, **kw)
+        self._args = tuple(t(v) if v is not None else None for t, v in zip(SIGNATURES[name][1], raw))
+        self._keep = tensors
+
+    def __call__(self) -> None:
+        st = self._fn(*self._args)
+        if st:
+            raise I8Error(st, self.name)
+
+    def with_stream(self, stream) -> "Prepared":
+        """The same call on another stream (the stream is the last argument of every compute entry point)."""
+        other = object.__new__(Prepared)
+        other.name, other._fn, other._keep = self.name, self._fn, self._keep
+        other._args = self._args[:-1] + (_vp(_stream_ptr(stream)),)
+        return other
+
+
+def prepare(name: str, *tensors, **kw) -> Prepared:
+    return Prepared(name, *tensors, **kw)
 
 
 def gemm_i8_host(A, B, C, bias, mult, shift, per_channel: int, relu: int, stream=None) -> None:
@@ -179,8 +223,8 @@ def mpc_forward_f32(Adyn, Bdyn, Kinf, x0, d, u, xs=None, stream=None) -> None:
 
 
 class Plan(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int) for n in ("shape_class", "tile_m", "tile_n", "stages", "m_tiles", "n_tiles", "waves",
-                                             "b_resident", "epilogue_warps")]
+    _fields_ = [(n, ctypes.c_int) for n in ("shape_class", "tile_m", "tile_n", "stages", "cta_group", "raster_group", "sticky",
+                                             "m_tiles", "n_tiles", "workers", "waves", "b_resident", "epilogue_warps")]
 
 
 def plan_gemm(M: int, N: int, K: int, sm_count: int = 148) -> dict:
@@ -190,8 +234,50 @@ def plan_gemm(M: int, N: int, K: int, sm_count: int = 148) -> dict:
     return {n: getattr(pl, n) for n, _ in Plan._fields_}
 
 
+def last_plan() -> dict:
+    """The plan of this thread's most recent launch of the large-tile tensor kernel."""
+    pl = Plan()
+    _check(lib().i8ops_last_plan(ctypes.byref(pl)), "i8ops_last_plan")
+    return {n: getattr(pl, n) for n, _ in Plan._fields_}
+
+
 def set_class_tile(shape_class: int, tile_n: int) -> None:
     _check(lib().i8ops_set_class_tile(int(shape_class), int(tile_n)), "i8ops_set_class_tile")
+
+
+def set_class_plan(shape_class: int, base=(0, 0, 0), tile_n: int = 0, cta_group: int = 0, raster_group: int = 0,
+                   sticky: int = -1) -> None:
+    """Record a schedule for a shape class (see ``i8ops_set_class_plan``); all defaults forgets the entry."""
+    _check(lib().i8ops_set_class_plan(int(shape_class), int(base[0]), int(base[1]), int(base[2]), int(tile_n), int(cta_group),
+                                      int(raster_group), int(sticky)), "i8ops_set_class_plan")
+
+
+def tmap_cache_stats():
+    """(hits, misses) of the calling thread's tensor-map cache."""
+    h, m = ctypes.c_uint64(0), ctypes.c_uint64(0)
+    _check(lib().i8ops_tmap_cache_stats(ctypes.byref(h), ctypes.byref(m)), "i8ops_tmap_cache_stats")
+    return int(h.value), int(m.value)
+
+
+def probe_mma_rate(tile_n: int = 256, reps: int = 8192, ctas: Optional[int] = None, stream=None) -> dict:
+    """Run the tensor-core issue-rate probe on `ctas` SMs (default: all) and return the measured int8 peak:
+    ``tops`` (whole chip, from the slowest CTA's wall time), ``cycles_per_mma`` (median over CTAs), ``sm_mhz`` (SM cycles per
+    nanosecond during the probe) and ``us`` (duration)."""
+    import torch
+    if ctas is None:
+        ctas = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    out = torch.zeros((ctas, 4), dtype=torch.int64, device="cuda")
+    _check(lib().i8ops_probe_mma_rate(int(tile_n), int(reps), int(ctas), _ptr(out), _stream_ptr(stream)), "i8ops_probe_mma_rate")
+    torch.cuda.synchronize()
+    o = out.cpu().numpy()
+    if (o[:, 2] == 0).any():
+        raise I8Error(8, "i8ops_probe_mma_rate")
+    ns = float(o[:, 2].max())
+    ops = float(ctas) * reps * 2.0 * 128 * tile_n * 32
+    cyc = sorted(o[:, 1].tolist())[ctas // 2]
+    return {"tile_n": tile_n, "reps": reps, "ctas": ctas, "tops": ops / ns / 1e3, "cycles_per_mma": cyc / reps,
+            "sm_mhz": cyc / float(sorted(o[:, 2].tolist())[ctas // 2]) * 1e3, "us": ns / 1e3,
+            "distinct_sms": int(len(set(o[:, 3].tolist())))}
 
 
 def last_device_status(stream=None) -> int:

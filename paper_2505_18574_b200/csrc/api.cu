@@ -6,6 +6,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 #include <utility>
 
@@ -15,6 +16,7 @@
 #include "gemm_tc.cuh"
 #include "generic.cuh"
 #include "mpc.cuh"
+#include "probe.cuh"
 
 namespace i8 {
 
@@ -24,14 +26,15 @@ __device__ unsigned g_dev_status = 0;   // first bounded-wait expiry since the l
 constexpr int MAX_DEVICES = 64;
 
 struct DeviceCtx {
-    bool ready = false;
+    std::atomic<bool> ready{false};   // set last (release) by the one-time set-up; read without the lock afterwards
     int sm_count = 0;
     unsigned* dev_status = nullptr;   // device address of g_dev_status
-    bool attr_set[16] = {};           // dynamic shared-memory opt-in done, per kernel instance
+    bool attr_set[32] = {};            // dynamic shared-memory opt-in done, per kernel instance
     void* ws = nullptr;               // workspace of the host-buffer variants
     size_t ws_bytes = 0;
     cudaStream_t s_in = nullptr, s_out = nullptr;   // copy streams of the host-buffer variants
     cudaEvent_t ev[2 * 8 + 2] = {};                 // chunk hand-over events (up to 8 row chunks)
+    std::mutex host_mutex;                          // serialises the host-buffer variant: its calls share ws, s_in, s_out and ev
 };
 
 static DeviceCtx g_ctx[MAX_DEVICES];
@@ -44,11 +47,13 @@ static int g_conv_two_sm = -1;                   // CTA pairs for convolutions: 
 static int g_force_bn = -1;                      // tuning override from the environment (I8OPS_FORCE_BN)
 static int g_tma_store = 1;                      // read-out of the wide tiles through TMA stores (I8OPS_TMA_STORE=0 turns it off)
 static int g_sticky = 1;                         // column-sticky tile order for short-K problems (I8OPS_STICKY=0 turns it off)
+static int g_tmap_cache = 1;                     // per-thread cache of encoded tensor maps (I8OPS_TMAP_CACHE=0 encodes every time)
 static int g_slab = 1;                           // slab-resident stride-1 convolution kernel (I8OPS_SLAB=0 turns it off)
 
 static thread_local int t_last_path = I8_PATH_NONE;
 static thread_local int t_last_cuda = 0;
 static thread_local bool t_used_two_sm = false;
+static thread_local bool t_tmap_failed = false;   // the last tensor-path attempt stopped at a tensor-map encoding (nothing launched)
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -76,9 +81,10 @@ static int get_ctx(DeviceCtx** out) {
     int dev = 0;
     CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= MAX_DEVICES) return cuda_fail(cudaErrorInvalidDevice);
-    std::lock_guard<std::mutex> lock(g_mutex);
     DeviceCtx& c = g_ctx[dev];
-    if (!c.ready) {
+    if (c.ready.load(std::memory_order_acquire)) { *out = &c; return I8_OK; }   // the hot path takes no lock
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!c.ready.load(std::memory_order_relaxed)) {
         CUDA_TRY(cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, dev));
         CUDA_TRY(cudaGetSymbolAddress((void**)&c.dev_status, g_dev_status));
         if (!g_encode_tiled) {
@@ -104,26 +110,106 @@ static int get_ctx(DeviceCtx** out) {
         if (sticky) g_sticky = atoi(sticky);
         const char* slab = getenv("I8OPS_SLAB");
         if (slab) g_slab = atoi(slab);
+        const char* tmc = getenv("I8OPS_TMAP_CACHE");
+        if (tmc) g_tmap_cache = atoi(tmc);
         const char* pdl = getenv("I8OPS_PDL");
         if (pdl) g_pdl = atoi(pdl);
-        c.ready = true;
+        c.ready.store(true, std::memory_order_release);
     }
     *out = &c;
     return I8_OK;
 }
 
-// 2-D or 3-D byte tensor, innermost dimension contiguous, 128-byte swizzle, zero fill outside.
-static int make_tmap(CUtensorMap* tm, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                     const uint32_t* box, CUtensorMapSwizzle swz) {
+// ------------------------------------------------------------------------------------------------ tensor maps
+// Encoding a tensor map is a driver call of about a microsecond, and a call needs two or three of them, which is as
+// much as a small problem's kernel time.  Maps depend only on the base address and the geometry, so each host thread
+// keeps the ones it encoded in a small direct-mapped cache (no lock: the cache is thread-local) keyed on everything
+// that goes into the encoding, the base pointer included.
+struct TmapKey {
+    uint64_t base;
+    uint64_t dims[5];
+    uint64_t strides[4];
+    uint32_t box[5];
+    uint32_t rank, swizzle, kind;     // kind: 0 tiled, 1 im2col
+    int32_t lower[2], upper[2];       // im2col: bounding-box corners
+    uint32_t estr[5];                 // traversal strides
+    uint32_t channels, pixels;        // im2col: channels per pixel, pixels per column
+};
+struct TmapEntry {
+    TmapKey key;
+    alignas(64) CUtensorMap map;
+    bool valid;
+};
+constexpr int TMAP_CACHE_SLOTS = 64;
+static thread_local TmapEntry t_tmap_cache[TMAP_CACHE_SLOTS];
+static thread_local uint64_t t_tmap_hits = 0, t_tmap_misses = 0;
+
+static uint32_t tmap_hash(const TmapKey& k) {
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(&k);
+    uint32_t h = 2166136261u;
+    for (size_t i = 0; i < sizeof(TmapKey) / 4; i++) h = (h ^ w[i]) * 16777619u;
+    return h ^ (h >> 15);
+}
+
+static int encode_tmap(CUtensorMap* tm, const TmapKey& k) {
     cuuint64_t gdim[5], gstr[4];
     cuuint32_t bx[5], es[5];
-    for (int i = 0; i < rank; i++) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
-    for (int i = 0; i + 1 < rank; i++) gstr[i] = strides_bytes[i];
-    CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bx, es,
-                                CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { t_last_cuda = (int)cudaErrorInvalidValue; return I8_ERR_CUDA; }
+    for (uint32_t i = 0; i < k.rank; i++) { gdim[i] = k.dims[i]; bx[i] = k.box[i]; es[i] = k.estr[i]; }
+    for (uint32_t i = 0; i + 1 < k.rank; i++) gstr[i] = k.strides[i];
+    CUresult r;
+    if (k.kind == 0)
+        r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, k.rank, reinterpret_cast<void*>(k.base), gdim, gstr, bx, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, (CUtensorMapSwizzle)k.swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    else
+        r = g_encode_im2col(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, k.rank, reinterpret_cast<void*>(k.base), gdim, gstr, k.lower, k.upper,
+                            k.channels, k.pixels, es, CU_TENSOR_MAP_INTERLEAVE_NONE, (CUtensorMapSwizzle)k.swizzle,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { t_last_cuda = (int)cudaErrorInvalidValue; t_tmap_failed = true; return I8_ERR_CUDA; }
     return I8_OK;
+}
+
+static int cached_tmap(CUtensorMap* tm, const TmapKey& k) {
+    if (!g_tmap_cache) return encode_tmap(tm, k);
+    TmapEntry& e = t_tmap_cache[tmap_hash(k) % TMAP_CACHE_SLOTS];
+    if (e.valid && memcmp(&e.key, &k, sizeof(TmapKey)) == 0) {
+        *tm = e.map;
+        t_tmap_hits++;
+        return I8_OK;
+    }
+    t_tmap_misses++;
+    int rc = encode_tmap(tm, k);
+    if (rc) return rc;
+    e.key = k; e.map = *tm; e.valid = true;
+    return I8_OK;
+}
+
+// Tiled byte tensor of rank 2..5, innermost dimension contiguous, zero fill outside.
+static int make_tmap(CUtensorMap* tm, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                     const uint32_t* box, CUtensorMapSwizzle swz) {
+    TmapKey k;
+    memset(&k, 0, sizeof(k));
+    k.base = reinterpret_cast<uint64_t>(base);
+    k.rank = (uint32_t)rank; k.swizzle = (uint32_t)swz; k.kind = 0;
+    for (int i = 0; i < rank; i++) { k.dims[i] = dims[i]; k.box[i] = box[i]; k.estr[i] = 1; }
+    for (int i = 0; i + 1 < rank; i++) k.strides[i] = strides_bytes[i];
+    return cached_tmap(tm, k);
+}
+
+// im2col-mode map over dense NHWC activations: `channels` bytes x `pixels` output positions per load.
+static int make_tmap_im2col(CUtensorMap* tm, const void* x, int N, int H, int W, int C, int R, int S, int stride_h, int stride_w,
+                            int pad_h, int pad_w, int channels, int pixels, CUtensorMapSwizzle swz) {
+    TmapKey k;
+    memset(&k, 0, sizeof(k));
+    k.base = reinterpret_cast<uint64_t>(x);
+    k.rank = 4; k.swizzle = (uint32_t)swz; k.kind = 1;
+    k.dims[0] = (uint64_t)C; k.dims[1] = (uint64_t)W; k.dims[2] = (uint64_t)H; k.dims[3] = (uint64_t)N;
+    k.strides[0] = (uint64_t)C; k.strides[1] = (uint64_t)W * C; k.strides[2] = (uint64_t)H * W * C;
+    k.lower[0] = -pad_w; k.lower[1] = -pad_h;
+    k.upper[0] = pad_w - (S - 1); k.upper[1] = pad_h - (R - 1);
+    k.estr[0] = 1; k.estr[1] = (uint32_t)stride_w; k.estr[2] = (uint32_t)stride_h; k.estr[3] = 1;
+    k.channels = (uint32_t)channels; k.pixels = (uint32_t)pixels;
+    return cached_tmap(tm, k);
 }
 
 // Launch on `st`; with programmatic stream serialisation the kernel may be scheduled while its predecessor in
@@ -180,11 +266,7 @@ static int launch_tc(DeviceCtx* ctx, int slot, const CUtensorMap& tmA, const CUt
     return I8_OK;
 }
 
-// Tile width.  Cost model in SM cycles: every wave of tiles pays, per 128-byte K block, an operand-delivery
-// bound of 256 + 2*BN, plus a fixed 400 per tile; the last tile's read-out (about 14 cycles per column) is
-// exposed.  The width with the lowest total wins; ties go to the wider tile.
-static int g_class_bn[3] = {0, 0, 0};            // per shape class: tile width recorded for reuse (0 = use the model)
-
+// ------------------------------------------------------------------------------------------------ planning
 // Shape classes of the paper's schedule-reuse experiment: a schedule found for one shape is reused for shapes of the
 // same aspect class (square, column-dominant = tall and narrow, row-dominant = short and wide).
 static int shape_class(int M, int N) {
@@ -193,9 +275,40 @@ static int shape_class(int M, int N) {
     return 0;
 }
 
-static int choose_bn(int M, int N, int num_kb, int sm_count) {
+// One recorded schedule per class: the choices the planner would otherwise take from its cost model.  An entry with a
+// base shape applies to shapes whose M, N and K each lie within a factor of four of the base's (the "nearby shapes" of
+// the paper's reuse table); an entry without one (base_m == 0) applies to the whole class.
+struct ClassPlan {
+    int valid;
+    int base_m, base_n, base_k;
+    int tile_n;          // 64, 128, 256; 0 = cost model
+    int cta_group;       // 1, 2; 0 = crossover rule
+    int raster_group;    // block rows per raster group; 0 = default
+    int sticky;          // 1 = column-sticky order where legal, 0 = never, -1 = rule
+};
+// Seeds: the tuned plans of the two workload configurations with a clear class (8192^3 on CTA pairs with 16-row raster
+// groups; the 262144 x 64 x 256 stream on 64-wide tiles with B resident).
+static ClassPlan g_class_plan[3] = {
+    {1, 8192, 8192, 8192, 256, 2, 16, -1},
+    {1, 262144, 64, 256, 64, 1, 16, -1},
+    {0, 0, 0, 0, 0, 0, 0, -1},
+};
+
+static bool near_base(int v, int base) { return (int64_t)v * 4 >= base && (int64_t)v <= (int64_t)base * 4; }
+
+static const ClassPlan* recorded_plan(int M, int N, int K) {
+    const ClassPlan& e = g_class_plan[shape_class(M, N)];
+    if (!e.valid) return nullptr;
+    if (e.base_m && !(near_base(M, e.base_m) && near_base(N, e.base_n) && near_base(K, e.base_k))) return nullptr;
+    return &e;
+}
+
+// Tile width.  Cost model in SM cycles: every wave of tiles pays, per 128-byte K block, an operand-delivery
+// bound of 256 + 2*BN, plus a fixed 400 per tile; the last tile's read-out (about 14 cycles per column) is
+// exposed.  The width with the lowest total wins; ties go to the wider tile.
+static int choose_bn(int M, int N, int num_kb, int sm_count, const ClassPlan* rec) {
     if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256) return g_force_bn;
-    const int recorded = g_class_bn[shape_class(M, N)];
+    const int recorded = rec ? rec->tile_n : 0;
     if (recorded && (recorded == 64 || recorded - 64 < ((N + 63) / 64) * 64)) return recorded;
     const int cands[3] = {256, 128, 64};
     int best = 64;
@@ -212,18 +325,91 @@ static int choose_bn(int M, int N, int num_kb, int sm_count) {
     return best;
 }
 
+// Everything the host decides about one launch of the large-tile kernel.  The launch code and the plan query both get
+// it from plan_tc(), so the query reports what runs.
+struct TcPlan {
+    int two_sm, bn, stages, tile_m;
+    int workers;                 // CTAs (one-SM) or CTA pairs launched
+    int m_tiles, n_tiles, num_tiles;
+    int group_m, sticky, col_base, col_rem;
+    int b_resident;
+    int shape_cls;
+};
+static thread_local TcPlan t_last_plan = {};
+
+// CTA pairs: their larger tiles and cluster set-up cost about 1.5 us more per launch, which pays once there is at least
+// one full wave of 256-row tiles and enough K per cluster (measured crossover: waves x K blocks ~ 48).
+static bool pair_pays(int M, int N, int bn, int num_kb, int sm_count) {
+    const int clusters = sm_count / 2;
+    const int64_t tiles2 = (int64_t)((M + 255) / 256) * ((N + bn - 1) / bn);
+    const int64_t waves2 = (tiles2 + clusters - 1) / clusters;
+    return tiles2 >= clusters && waves2 * num_kb >= 48;
+}
+
+// conv: the operand A comes through im2col loads (three two-SM instances exist); GEMM: the two-SM instance is 256 wide.
+// num_kb = 128-byte K blocks, num_iters = ring slots per tile, cb = bytes of K per sub-block.
+static TcPlan plan_tc(bool conv, int M, int N, int K, int num_kb, int num_iters, int num_kblocks, int cb, int sm_count) {
+    TcPlan pl = {};
+    pl.shape_cls = shape_class(M, N);
+    const ClassPlan* rec = conv ? nullptr : recorded_plan(M, N, K);
+    bool two_sm;
+    int bn;
+    if (conv) {
+        bn = choose_bn(M, N, num_kb, sm_count, nullptr);
+        two_sm = g_path_mode == 2 || g_conv_two_sm == 1;
+        if (g_tc2 && g_conv_two_sm != 0 && g_force_bn < 0 && pair_pays(M, N, bn, num_kb, sm_count)) two_sm = true;
+    } else {
+        bool want2 = g_tc2 && pair_pays(M, N, 256, num_kb, sm_count);
+        if (rec && rec->cta_group == 1) want2 = false;
+        if (rec && rec->cta_group == 2 && g_tc2) want2 = true;
+        two_sm = g_force_bn < 0 && (want2 || g_path_mode == 2);
+        bn = two_sm ? 256 : choose_bn(M, N, num_kb, sm_count, rec);
+    }
+    pl.two_sm = two_sm ? 1 : 0;
+    pl.bn = bn;
+    pl.tile_m = two_sm ? 2 * BM : BM;
+    // ring slots per instance (must match the launch table in run_tc)
+    // (64-wide GEMM tiles: 6 slots measured 4 % faster than 8 on the tall-skinny stream, as deep rings also were on the batched kernel)
+    pl.stages = two_sm ? (bn == 256 ? 6 : 8) : (bn == 256 ? 4 : (bn == 128 ? 6 : (conv ? 8 : 6)));
+    pl.m_tiles = (M + pl.tile_m - 1) / pl.tile_m;
+    pl.n_tiles = (N + bn - 1) / bn;
+    pl.num_tiles = pl.m_tiles * pl.n_tiles;
+    const int max_workers = two_sm ? sm_count / 2 : sm_count;
+    pl.workers = pl.num_tiles < max_workers ? pl.num_tiles : max_workers;
+    pl.group_m = (rec && rec->raster_group > 0) ? rec->raster_group : 16;   // 16: measured best of 2..32 on 8192^3 for the two-SM kernel
+    // Column-sticky order for short-K problems with several tiles per worker: rebuilding the epilogue constants for
+    // a new block column costs about as much as a short tile, so a worker keeps its column if that needs no more
+    // rounds than the raster order.
+    pl.sticky = 0; pl.col_base = 0; pl.col_rem = 0;
+    {
+        const int nt = pl.n_tiles, mt = pl.m_tiles, workers = max_workers;
+        const int pref = rec ? rec->sticky : -1;
+        const bool legal = nt > 1 && workers >= 2 * nt && pl.num_tiles > workers;
+        if (g_sticky && legal && pref != 0 && (pref == 1 || num_iters <= 16)) {
+            const int base = workers / nt;
+            const int rounds_sticky = (mt + base - 1) / base;
+            const int rounds_raster = (pl.num_tiles + workers - 1) / workers;
+            if (pref == 1 || rounds_sticky <= rounds_raster) { pl.sticky = 1; pl.col_base = base; pl.col_rem = workers % nt; }
+        }
+    }
+    // resident B: one block column, and all of B's K blocks fit the ring's B region
+    const int b_rows = two_sm ? bn / 2 : bn;
+    pl.b_resident = (pl.n_tiles == 1 && (int64_t)num_kblocks * b_rows * cb <= (int64_t)pl.stages * b_rows * BK) ? 1 : 0;
+    return pl;
+}
+
 // Common tail of the tensor paths: B's tensor map (an N x K matrix with K contiguous), the tile schedule,
 // and the launch of the instance that matches the tile width.
 struct RawOut { int32_t* D = nullptr; int64_t ldd = 0; int accumulate = 0; };
 
-static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA, const KLoop& kl, int bn, const int8_t* B,
+static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap& tmA, const KLoop& kl, const int8_t* B,
                   int64_t ldb, int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult, const int32_t* shift,
                   int per_channel, int M, int N, int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
+    const bool two_sm = pl.two_sm != 0;
+    const int bn = pl.bn;
     const int b_rows = two_sm ? bn / 2 : bn;           // rows of the B tile one CTA loads
-    const int tile_m = two_sm ? 2 * BM : BM;
-    // ring slots per instance (must match the launch table below)
-    // (64-wide GEMM tiles: 6 slots measured 4 % faster than 8 on the tall-skinny stream, as deep rings also were on the batched kernel)
-    const int stages = two_sm ? (bn == 256 ? 6 : 8) : (bn == 256 ? 4 : (bn == 128 ? 6 : (conv ? 8 : 6)));
+    t_last_plan = pl;
+    t_used_two_sm = two_sm;
     CUtensorMap tmB;
     {
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
@@ -250,42 +436,24 @@ static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA
         if (rc) return rc;
         p.tma_store = 1;
     }
-    p.sched.m_tiles = (M + tile_m - 1) / tile_m;
-    p.sched.n_tiles = (N + bn - 1) / bn;
-    p.sched.num_tiles = p.sched.m_tiles * p.sched.n_tiles;
-    p.sched.group_m = 16;                              // measured best of 2..32 on 8192^3 for the two-SM kernel
-    p.sched.sticky = 0; p.sched.col_base = 0; p.sched.col_rem = 0;
+    p.sched.m_tiles = pl.m_tiles;
+    p.sched.n_tiles = pl.n_tiles;
+    p.sched.num_tiles = pl.num_tiles;
+    p.sched.group_m = pl.group_m;
+    p.sched.sticky = pl.sticky; p.sched.col_base = pl.col_base; p.sched.col_rem = pl.col_rem;
     {
         auto inv32 = [](int d) { return d <= 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)d); };
-        const int workers = two_sm ? ctx->sm_count / 2 : ctx->sm_count;
         p.sched.inv_nt = inv32(p.sched.n_tiles);
         p.sched.inv_width = inv32(p.sched.group_m * p.sched.n_tiles);
         p.sched.inv_gm = inv32(p.sched.group_m);
-        p.sched.inv_step = inv32(p.sched.num_tiles < workers ? p.sched.num_tiles : workers);
+        p.sched.inv_step = inv32(pl.workers);
         const int last = p.sched.m_tiles % p.sched.group_m;
         p.sched.inv_last = inv32(last ? last : p.sched.group_m);
-        p.sched.inv_cb = 0xffffffffu; p.sched.inv_cb1 = 0xffffffffu;
-    }
-    {
-        // Column-sticky order for short-K problems with several tiles per worker: rebuilding the epilogue constants for
-        // a new block column costs about as much as a short tile, so a worker keeps its column if that needs no more
-        // rounds than the raster order.
-        const int workers = two_sm ? ctx->sm_count / 2 : ctx->sm_count;
-        const int nt = p.sched.n_tiles, mt = p.sched.m_tiles;
-        if (g_sticky && nt > 1 && workers >= 2 * nt && p.sched.num_tiles > workers && kl.num_iters <= 16) {
-            const int base = workers / nt;
-            const int rounds_sticky = (mt + base - 1) / base;
-            const int rounds_raster = (p.sched.num_tiles + workers - 1) / workers;
-            if (rounds_sticky <= rounds_raster) {
-                p.sched.sticky = 1; p.sched.col_base = base; p.sched.col_rem = workers % nt;
-                p.sched.inv_cb = base <= 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)base);
-                p.sched.inv_cb1 = (uint32_t)((1ull << 32) / (uint64_t)(base + 1));
-            }
-        }
+        p.sched.inv_cb = pl.sticky ? inv32(pl.col_base) : 0xffffffffu;
+        p.sched.inv_cb1 = pl.sticky ? inv32(pl.col_base + 1) : 0xffffffffu;
     }
     p.kl = kl;
-    // resident B: one block column, and all of B's K blocks fit the ring's B region
-    p.kl.b_resident = (p.sched.n_tiles == 1 && (int64_t)kl.num_kblocks * b_rows * kl.cb <= (int64_t)stages * b_rows * BK) ? 1 : 0;
+    p.kl.b_resident = pl.b_resident;
     p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);   // SM clock stays below 2 GHz: at least the asked time
     p.dev_status = ctx->dev_status;
     if (two_sm) {
@@ -312,32 +480,26 @@ static int run_tc(DeviceCtx* ctx, bool conv, bool two_sm, const CUtensorMap& tmA
     }
 }
 
+static KLoop gemm_kloop(int K) {
+    KLoop kl{};
+    kl.cb = BK; kl.nsub = 1; kl.num_kblocks = (K + BK - 1) / BK;
+    kl.num_iters = kl.num_kblocks;
+    kl.mmas_last = ((K - (kl.num_iters - 1) * BK) + 31) / 32;
+    return kl;
+}
+
 static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
                        int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
-    // two-SM kernel: its larger tiles and cluster set-up cost about 1.5 us more per launch, which pays once there
-    // is at least one full wave of 256 x 256 tiles and enough K per cluster (measured crossover: waves x K blocks ~ 48)
-    bool two_sm = false;
-    {
-        const int clusters = ctx->sm_count / 2;
-        const int64_t tiles2 = (int64_t)((M + 255) / 256) * ((N + 255) / 256);
-        const int64_t waves2 = (tiles2 + clusters - 1) / clusters;
-        const bool big = tiles2 >= clusters && waves2 * ((K + BK - 1) / BK) >= 48;
-        two_sm = g_force_bn < 0 && ((g_tc2 && big) || g_path_mode == 2);
-    }
-    t_used_two_sm = two_sm;
-    const int bn = two_sm ? 256 : choose_bn(M, N, (K + BK - 1) / BK, ctx->sm_count);
+    const KLoop kl = gemm_kloop(K);
+    const TcPlan pl = plan_tc(false, M, N, K, kl.num_kblocks, kl.num_iters, kl.num_kblocks, BK, ctx->sm_count);
     CUtensorMap tmA;
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
     const uint64_t str[1] = {(uint64_t)lda};
     const uint32_t box[2] = {BK, BM};
     int rc = make_tmap(&tmA, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
-    KLoop kl{};
-    kl.cb = BK; kl.nsub = 1; kl.num_kblocks = (K + BK - 1) / BK;
-    kl.num_iters = kl.num_kblocks;
-    kl.mmas_last = ((K - (kl.num_iters - 1) * BK) + 31) / 32;
-    return run_tc(ctx, false, two_sm, tmA, kl, bn, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
+    return run_tc(ctx, false, pl, tmA, kl, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
 }
 
 // Implicit-GEMM convolution: A tiles come from an im2col-mode tensor map over the NHWC activations.
@@ -346,28 +508,10 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
                        int stride_h, int stride_w, int pad_h, int pad_w, int relu, cudaStream_t st) {
     const int cb = C % 128 == 0 ? 128 : (C % 64 == 0 ? 64 : 32);
     const int M = N * P * Q;
-    const int bn = choose_bn(M, Kf, (R * S * C + BK - 1) / BK, ctx->sm_count);
-    // CTA pairs for convolutions: the same measured rule as for GEMMs (a full wave of 256-row tiles and enough K per
-    // cluster to amortise the pair's extra set-up), or asked for explicitly (path mode 2, I8OPS_CONV2SM=1)
-    bool two_sm = g_path_mode == 2 || g_conv_two_sm == 1;
-    if (g_tc2 && g_conv_two_sm != 0 && g_force_bn < 0) {
-        const int clusters = ctx->sm_count / 2;
-        const int64_t tiles2 = (int64_t)((M + 255) / 256) * ((Kf + bn - 1) / bn);
-        const int64_t waves2 = (tiles2 + clusters - 1) / clusters;
-        if (tiles2 >= clusters && waves2 * ((R * S * C + BK - 1) / BK) >= 48) two_sm = true;
-    }
-    t_used_two_sm = two_sm;
     CUtensorMap tmA;
     {
-        const cuuint64_t gdim[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
-        const cuuint64_t gstr[3] = {(cuuint64_t)C, (cuuint64_t)W * C, (cuuint64_t)H * W * C};
-        const int lower[2] = {-pad_w, -pad_h};
-        const int upper[2] = {pad_w - (S - 1), pad_h - (R - 1)};
-        const cuuint32_t estr[4] = {1, (cuuint32_t)stride_w, (cuuint32_t)stride_h, 1};
-        CUresult r = g_encode_im2col(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(x), gdim, gstr, lower, upper,
-                                     (cuuint32_t)cb, (cuuint32_t)BM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(cb),
-                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) { t_last_cuda = (int)cudaErrorInvalidValue; return I8_ERR_CUDA; }
+        int rc = make_tmap_im2col(&tmA, x, N, H, W, C, R, S, stride_h, stride_w, pad_h, pad_w, cb, BM, swizzle_for(cb));
+        if (rc) return rc;
     }
     KLoop kl{};
     kl.cb = cb; kl.nsub = BK / cb; kl.cblocks = C / cb; kl.num_kblocks = R * S * kl.cblocks;
@@ -378,7 +522,9 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     kl.mmas_last = (kl.num_kblocks - (kl.num_iters - 1) * kl.nsub) * (cb / 32);
     kl.stride_h = stride_h; kl.stride_w = stride_w; kl.pad_h = pad_h; kl.pad_w = pad_w;
     const int K = R * S * C;
-    return run_tc(ctx, true, two_sm, tmA, kl, bn, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
+    // CTA pairs for convolutions follow the same measured rule as for GEMMs, or are asked for explicitly (path mode 2, I8OPS_CONV2SM=1)
+    const TcPlan pl = plan_tc(true, M, Kf, K, (K + BK - 1) / BK, kl.num_iters, kl.num_kblocks, cb, ctx->sm_count);
+    return run_tc(ctx, true, pl, tmA, kl, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
 }
 
 // Slab-resident stride-1 convolution (conv_slab.cuh): plan and launch.  Returns I8_ERR_UNSUPPORTED, launching nothing,
@@ -537,10 +683,11 @@ int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_
     const bool tc_legal = K >= 1 && a_cs == 1 && b_rs == 1 && aligned16(A) && aligned16(B) && a_rs % 16 == 0 &&
                           b_cs % 16 == 0 && a_rs >= K && b_cs >= K;
     if (tc_legal && g_path_mode != 1) {
-        t_used_two_sm = false;
+        t_used_two_sm = false; t_tmap_failed = false;
         rc = run_gemm_tc(ctx, A, a_rs, B, b_cs, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
         if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
-        return rc;
+        if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
+        // the driver refused a tensor map for this geometry: nothing was launched, the generic kernel serves it
     }
     GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, C, ldc, 0, bias, 0, mult, shift, per_channel, relu, 1, M, N, K, nullptr, 0, 0, 0};
     rc = run_gemm_generic(g, st);
@@ -564,10 +711,10 @@ int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, in
                           b_cs % 16 == 0 && a_rs >= K && b_cs >= K;
     if (tc_legal && g_path_mode != 1) {
         RawOut raw; raw.D = D; raw.ldd = ldd; raw.accumulate = accumulate ? 1 : 0;
-        t_used_two_sm = false;
+        t_used_two_sm = false; t_tmap_failed = false;
         rc = run_gemm_tc(ctx, A, a_rs, B, b_cs, nullptr, 0, nullptr, nullptr, nullptr, 0, M, N, K, 0, st, raw);
         if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
-        return rc;
+        if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
     }
     GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, nullptr, 0, 0, nullptr, 0, nullptr, nullptr, 0, 0, 1, M, N, K,
                         D, ldd, 1, accumulate ? 1 : 0};
@@ -590,15 +737,17 @@ int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs, c
     rc = get_ctx(&ctx);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    // (an operand shared by all problems, batch stride 0, has no 3-D tensor map: the generic kernel serves it)
     if (g_path_mode != 1 && M <= 64 && N <= 64 && K >= 1 && K <= 64 && a_cs == 1 && aligned16(A) && aligned16(B) &&
-        a_rs % 16 == 0 && a_bs % 16 == 0 && b_bs % 16 == 0 && a_rs >= K) {
+        a_rs % 16 == 0 && a_bs % 16 == 0 && b_bs % 16 == 0 && a_rs >= K && (batch == 1 || (a_bs > 0 && b_bs > 0))) {
         const bool b_n_contig = b_cs == 1 && b_rs % 16 == 0 && b_rs >= N;      // row-major B: MN-major operand
         const bool b_k_contig = b_rs == 1 && b_cs % 16 == 0 && b_cs >= K;      // column-major B: K-major operand
         if (b_k_contig || b_n_contig) {
+            t_tmap_failed = false;
             rc = run_batched_pair(ctx, A, a_rs, a_bs, B, b_k_contig ? b_cs : b_rs, b_bs, b_k_contig ? 0 : 1, C, ldc, c_bs,
                                   bias, bias_bs, mult, shift, per_channel, batch, M, N, K, relu, st);
             if (rc == I8_OK) t_last_path = I8_PATH_SMALL;
-            return rc;
+            if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
     }
     GenericGemmParams g{A, a_rs, a_cs, a_bs, B, b_rs, b_cs, b_bs, C, ldc, c_bs, bias, bias_bs, mult, shift, per_channel, relu,
@@ -624,29 +773,31 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     if (g_path_mode != 1 && aligned16(x) && aligned16(w)) {
-        if (R == 1 && S == 1 && stride_h == 1 && stride_w == 1 && pad_h == 0 && pad_w == 0 && C % 16 == 0) {
+        if (R == 1 && S == 1 && stride_h == 1 && stride_w == 1 && pad_h == 0 && pad_w == 0 && C % 16 == 0 &&
+            (int64_t)N * H * W < (1ll << 31)) {
             // a 1x1 convolution is the GEMM [N*H*W, C] x [C, K]
-            t_used_two_sm = false;
+            t_used_two_sm = false; t_tmap_failed = false;
             rc = run_gemm_tc(ctx, x, C, w, C, y, K, bias, mult, shift, per_channel, N * H * W, K, C, relu, st);
             if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
-            return rc;
+            if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
         if (g_slab && g_path_mode == 0 && stride_h == 1 && stride_w == 1 && (int64_t)N * P * Q < (1ll << 31)) {
             // few filters and a narrow image: keep the input slab in shared memory and reuse it across the filter taps
+            t_tmap_failed = false;
             rc = run_conv_slab(ctx, x, w, y, bias, mult, shift, per_channel, N, H, W, C, K, R, S, P, Q, pad_h, pad_w, relu, st);
             if (rc == I8_OK) { t_last_path = I8_PATH_CONV_SLAB; return rc; }
-            if (rc != I8_ERR_UNSUPPORTED) return rc;
+            if (rc != I8_ERR_UNSUPPORTED && !(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
         // im2col tensor maps: channel blocks of 32/64/128 bytes, box corners and tap offsets within the 4-D
         // encoding's ranges, traversal strides up to 8; activation tensors below 128 KiB stay on the generic kernel
         const bool tc_legal = C % 32 == 0 && R <= 16 && S <= 16 && pad_h <= 16 && pad_w <= 16 && stride_h <= 8 &&
                               stride_w <= 8 && (int64_t)N * H * W * C >= 131072 && (int64_t)N * P * Q < (1ll << 31);
         if (tc_legal) {
-            t_used_two_sm = false;
+            t_used_two_sm = false; t_tmap_failed = false;
             rc = run_conv_tc(ctx, x, w, y, bias, mult, shift, per_channel, N, H, W, C, K, R, S, P, Q, stride_h, stride_w,
                              pad_h, pad_w, relu, st);
             if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
-            return rc;
+            if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
     }
     GenericConvParams g{x, w, y, bias, mult, shift, per_channel, relu, N, H, W, C, K, R, S, P, Q, stride_h, stride_w, pad_h, pad_w};
@@ -673,17 +824,18 @@ int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C, const int32_t* bia
     int rc = get_ctx(&ctx);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    // One call at a time per device: the workspace, the two copy streams and the events below belong to the device's
+    // context, so a second host thread waits here until the first call has synchronised and returned.
+    std::lock_guard<std::mutex> host_lock(ctx->host_mutex);
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
     const size_t szA = up((size_t)M * K), szB = up((size_t)N * K), szC = up((size_t)M * N);
     const size_t szV = up((size_t)N * 4);
     const size_t need = szA + szB + szC + 3 * szV;
-    {
-        std::lock_guard<std::mutex> lock(g_mutex);
-        if (ctx->ws_bytes < need) {
-            if (ctx->ws) { CUDA_TRY(cudaDeviceSynchronize()); CUDA_TRY(cudaFree(ctx->ws)); ctx->ws = nullptr; ctx->ws_bytes = 0; }
-            CUDA_TRY(cudaMalloc(&ctx->ws, need));
-            ctx->ws_bytes = need;
-        }
+    if (ctx->ws_bytes < need) {
+        // every earlier call synchronised before it returned, so nothing still uses the old workspace
+        if (ctx->ws) { CUDA_TRY(cudaFree(ctx->ws)); ctx->ws = nullptr; ctx->ws_bytes = 0; }
+        CUDA_TRY(cudaMalloc(&ctx->ws, need));
+        ctx->ws_bytes = need;
     }
     uint8_t* base = (uint8_t*)ctx->ws;
     int8_t* dA = (int8_t*)base; int8_t* dB = (int8_t*)(base + szA); int8_t* dC = (int8_t*)(base + szA + szB);
@@ -694,58 +846,62 @@ int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C, const int32_t* bia
     // overlap (the two copy directions use separate DMA engines), so the host link is busy in both directions.
     const int nchunks = (K > 0 && M >= 2048) ? (M >= 8192 ? 8 : 4) : 1;
     if (nchunks > 1 && !ctx->s_in) {
-        std::lock_guard<std::mutex> lock(g_mutex);
-        if (!ctx->s_in) {
-            CUDA_TRY(cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking));
-            for (auto& e : ctx->ev) CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-            CUDA_TRY(cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking));
-        }
+        CUDA_TRY(cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking));
+        for (auto& e : ctx->ev) CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        CUDA_TRY(cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking));
     }
+    // Whatever was queued before an error is allowed to finish before the call returns: the buffers are the caller's
+    // and the workspace may be handed to the next call.
+    auto drain = [&](int status) {
+        if (ctx->s_in) cudaStreamSynchronize(ctx->s_in);
+        if (ctx->s_out) cudaStreamSynchronize(ctx->s_out);
+        cudaStreamSynchronize(st);
+        return status;
+    };
+#define HOST_TRY(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) return drain(cuda_fail(_e)); } while (0)
     if (nchunks == 1) {
         if (K > 0) {
-            CUDA_TRY(cudaMemcpyAsync(dA, A, (size_t)M * K, cudaMemcpyHostToDevice, st));
-            CUDA_TRY(cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, st));
+            HOST_TRY(cudaMemcpyAsync(dA, A, (size_t)M * K, cudaMemcpyHostToDevice, st));
+            HOST_TRY(cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, st));
         }
-        if (bias) CUDA_TRY(cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, st));
-        CUDA_TRY(cudaMemcpyAsync(dmult, mult, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
-        CUDA_TRY(cudaMemcpyAsync(dshift, shift, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
+        if (bias) HOST_TRY(cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, st));
+        HOST_TRY(cudaMemcpyAsync(dmult, mult, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
+        HOST_TRY(cudaMemcpyAsync(dshift, shift, (size_t)nq * 4, cudaMemcpyHostToDevice, st));
         rc = gemm_i8(dA, K, 1, dB, 1, K, dC, N, bias ? dbias : nullptr, dmult, dshift, per_channel, M, N, K, relu, stream);
-        if (rc) return rc;
-        CUDA_TRY(cudaMemcpyAsync(C, dC, (size_t)M * N, cudaMemcpyDeviceToHost, st));
-        CUDA_TRY(cudaStreamSynchronize(st));
+        if (rc) return drain(rc);
+        HOST_TRY(cudaMemcpyAsync(C, dC, (size_t)M * N, cudaMemcpyDeviceToHost, st));
+        HOST_TRY(cudaStreamSynchronize(st));
         return I8_OK;
     }
     cudaEvent_t* ev_in = ctx->ev;            // [i]: chunk i of A (and, for i = 0, B and the vectors) is on the device
     cudaEvent_t* ev_k = ctx->ev + 8;         // [i]: the kernel of chunk i is done
     cudaEvent_t ev_start = ctx->ev[16], ev_done = ctx->ev[17];
-    CUDA_TRY(cudaEventRecord(ev_start, st)); // the copy streams start after whatever the caller queued on `stream`
-    CUDA_TRY(cudaStreamWaitEvent(ctx->s_in, ev_start, 0));
-    CUDA_TRY(cudaStreamWaitEvent(ctx->s_out, ev_start, 0));
-    CUDA_TRY(cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, ctx->s_in));
-    if (bias) CUDA_TRY(cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, ctx->s_in));
-    CUDA_TRY(cudaMemcpyAsync(dmult, mult, (size_t)nq * 4, cudaMemcpyHostToDevice, ctx->s_in));
-    CUDA_TRY(cudaMemcpyAsync(dshift, shift, (size_t)nq * 4, cudaMemcpyHostToDevice, ctx->s_in));
+    HOST_TRY(cudaEventRecord(ev_start, st)); // the copy streams start after whatever the caller queued on `stream`
+    HOST_TRY(cudaStreamWaitEvent(ctx->s_in, ev_start, 0));
+    HOST_TRY(cudaStreamWaitEvent(ctx->s_out, ev_start, 0));
+    HOST_TRY(cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, ctx->s_in));
+    if (bias) HOST_TRY(cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, ctx->s_in));
+    HOST_TRY(cudaMemcpyAsync(dmult, mult, (size_t)nq * 4, cudaMemcpyHostToDevice, ctx->s_in));
+    HOST_TRY(cudaMemcpyAsync(dshift, shift, (size_t)nq * 4, cudaMemcpyHostToDevice, ctx->s_in));
     const int rows_per = (((M + nchunks - 1) / nchunks) + 255) / 256 * 256;
-    int used = 0;
     for (int i = 0; i < nchunks; i++) {
         const int r0 = i * rows_per;
         if (r0 >= M) break;
         const int rows = M - r0 < rows_per ? M - r0 : rows_per;
-        CUDA_TRY(cudaMemcpyAsync(dA + (size_t)r0 * K, A + (size_t)r0 * K, (size_t)rows * K, cudaMemcpyHostToDevice, ctx->s_in));
-        CUDA_TRY(cudaEventRecord(ev_in[i], ctx->s_in));
-        CUDA_TRY(cudaStreamWaitEvent(st, ev_in[i], 0));
+        HOST_TRY(cudaMemcpyAsync(dA + (size_t)r0 * K, A + (size_t)r0 * K, (size_t)rows * K, cudaMemcpyHostToDevice, ctx->s_in));
+        HOST_TRY(cudaEventRecord(ev_in[i], ctx->s_in));
+        HOST_TRY(cudaStreamWaitEvent(st, ev_in[i], 0));
         rc = gemm_i8(dA + (size_t)r0 * K, K, 1, dB, 1, K, dC + (size_t)r0 * N, N, bias ? dbias : nullptr, dmult, dshift, per_channel,
                      rows, N, K, relu, stream);
-        if (rc) return rc;
-        CUDA_TRY(cudaEventRecord(ev_k[i], st));
-        CUDA_TRY(cudaStreamWaitEvent(ctx->s_out, ev_k[i], 0));
-        CUDA_TRY(cudaMemcpyAsync(C + (size_t)r0 * N, dC + (size_t)r0 * N, (size_t)rows * N, cudaMemcpyDeviceToHost, ctx->s_out));
-        used++;
+        if (rc) return drain(rc);
+        HOST_TRY(cudaEventRecord(ev_k[i], st));
+        HOST_TRY(cudaStreamWaitEvent(ctx->s_out, ev_k[i], 0));
+        HOST_TRY(cudaMemcpyAsync(C + (size_t)r0 * N, dC + (size_t)r0 * N, (size_t)rows * N, cudaMemcpyDeviceToHost, ctx->s_out));
     }
-    (void)used;
-    CUDA_TRY(cudaEventRecord(ev_done, ctx->s_out));
-    CUDA_TRY(cudaStreamWaitEvent(st, ev_done, 0));
-    CUDA_TRY(cudaStreamSynchronize(st));
+    HOST_TRY(cudaEventRecord(ev_done, ctx->s_out));
+    HOST_TRY(cudaStreamWaitEvent(st, ev_done, 0));
+    HOST_TRY(cudaStreamSynchronize(st));
+#undef HOST_TRY
     return I8_OK;
 }
 
@@ -814,28 +970,76 @@ int mpc_forward_f32(const float* Adyn, const float* Bdyn, const float* Kinf, con
     return I8_OK;
 }
 
+static void fill_plan(const TcPlan& pl, i8_plan* out) {
+    out->shape_class = pl.shape_cls;
+    out->tile_m = pl.tile_m;
+    out->tile_n = pl.bn;
+    out->stages = pl.stages;
+    out->cta_group = pl.two_sm ? 2 : 1;
+    out->raster_group = pl.group_m;
+    out->sticky = pl.sticky;
+    out->m_tiles = pl.m_tiles;
+    out->n_tiles = pl.n_tiles;
+    out->workers = pl.workers;
+    out->waves = pl.workers ? (pl.num_tiles + pl.workers - 1) / pl.workers : 0;
+    out->b_resident = pl.b_resident;
+    out->epilogue_warps = 8;
+}
+
 int i8ops_plan_gemm(int M, int N, int K, int sm_count, i8_plan* out) {
     if (!out) return I8_ERR_NULL;
     if (M <= 0 || N <= 0 || K <= 0 || sm_count <= 0) return I8_ERR_SHAPE;
-    const int num_kb = (K + BK - 1) / BK;
-    const int bn = choose_bn(M, N, num_kb, sm_count);
-    const int stages = bn == 256 ? 4 : 6;
-    out->shape_class = shape_class(M, N);
-    out->tile_m = BM;
-    out->tile_n = bn;
-    out->stages = stages;
-    out->m_tiles = (M + BM - 1) / BM;
-    out->n_tiles = (N + bn - 1) / bn;
-    out->waves = (int)(((int64_t)out->m_tiles * out->n_tiles + sm_count - 1) / sm_count);
-    out->b_resident = (out->n_tiles == 1 && (int64_t)num_kb * bn * BK <= (int64_t)stages * bn * BK) ? 1 : 0;
-    out->epilogue_warps = 8;
+    const KLoop kl = gemm_kloop(K);
+    fill_plan(plan_tc(false, M, N, K, kl.num_kblocks, kl.num_iters, kl.num_kblocks, BK, sm_count), out);
+    return I8_OK;
+}
+
+int i8ops_last_plan(i8_plan* out) {
+    if (!out) return I8_ERR_NULL;
+    fill_plan(t_last_plan, out);
+    return I8_OK;
+}
+
+int i8ops_set_class_plan(int shape_cls, int base_m, int base_n, int base_k, int tile_n, int cta_group, int raster_group, int sticky) {
+    if (shape_cls < 0 || shape_cls > 2) return I8_ERR_RANGE;
+    if (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) return I8_ERR_RANGE;
+    if (cta_group < 0 || cta_group > 2 || raster_group < 0 || raster_group > 64 || sticky < -1 || sticky > 1) return I8_ERR_RANGE;
+    if (base_m < 0 || base_n < 0 || base_k < 0 || ((base_m == 0) != (base_n == 0)) || ((base_m == 0) != (base_k == 0))) return I8_ERR_RANGE;
+    if (cta_group == 2 && tile_n != 0 && tile_n != 256) return I8_ERR_RANGE;      // the pair kernel for GEMMs is 256 wide
+    ClassPlan e = {1, base_m, base_n, base_k, tile_n, cta_group, raster_group, sticky};
+    if (tile_n == 0 && cta_group == 0 && raster_group == 0 && sticky == -1) e.valid = 0;   // nothing recorded: forget the entry
+    g_class_plan[shape_cls] = e;
     return I8_OK;
 }
 
 int i8ops_set_class_tile(int shape_cls, int tile_n) {
-    if (shape_cls < 0 || shape_cls > 2) return I8_ERR_RANGE;
-    if (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) return I8_ERR_RANGE;
-    g_class_bn[shape_cls] = tile_n;
+    return i8ops_set_class_plan(shape_cls, 0, 0, 0, tile_n, 0, 0, -1);
+}
+
+int i8ops_tmap_cache_stats(uint64_t* hits, uint64_t* misses) {
+    if (!hits || !misses) return I8_ERR_NULL;
+    *hits = t_tmap_hits;
+    *misses = t_tmap_misses;
+    return I8_OK;
+}
+
+int i8ops_probe_mma_rate(int tile_n, int reps, int ctas, unsigned long long* out, void* stream) {
+    if (!out) return I8_ERR_NULL;
+    if (tile_n < 16 || tile_n > 256 || tile_n % 16 != 0 || reps < 64 || reps % 64 != 0 || reps > (1 << 24) || ctas < 1) return I8_ERR_RANGE;
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    if (ctas > ctx->sm_count) return I8_ERR_RANGE;            // one CTA per SM: more would share tensor cores
+    if (!ctx->attr_set[20]) {
+        CUDA_TRY(cudaFuncSetAttribute(mma_issue_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROBE_SMEM));
+        ctx->attr_set[20] = true;
+    }
+    MmaProbeParams p;
+    p.n = tile_n; p.reps = reps; p.out = out;
+    p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);
+    p.dev_status = ctx->dev_status;
+    mma_issue_probe_kernel<<<ctas, PROBE_THREADS, PROBE_SMEM, (cudaStream_t)stream>>>(p);
+    CUDA_TRY(cudaGetLastError());
     return I8_OK;
 }
 
@@ -853,7 +1057,7 @@ void i8ops_set_wait_limit_ms(int ms) {
     g_wait_limit_ns = (uint64_t)ms * 1000ull * 1000ull;
 }
 
-int i8ops_version(void) { return 1; }
+int i8ops_version(void) { return 2; }
 
 }  // extern "C"
 

@@ -41,16 +41,6 @@ def gemm_oracle(p):
     return C[:, :p.N]
 
 
-def gemm_oracle_rows(p, rows):
-    """Oracle result for a subset of rows of a row-major-A problem (used at sizes too large to do in full)."""
-    import oracle
-    assert p.a_cs == 1
-    As = np.ascontiguousarray(p.A[rows])
-    C = oracle.gemm_i8(As, p.a_rs, 1, p.B, p.b_rs, p.b_cs, p.N, p.bias, p.mult, p.shift, p.per_channel,
-                       len(rows), p.N, p.K, p.relu)
-    return C
-
-
 # ------------------------------------------------------------------------------------------------ batched
 def batched_gpu(p):
     import torch

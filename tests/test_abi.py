@@ -108,7 +108,16 @@ def test_tile_plan_and_class_reuse(L):
             assert pl["m_tiles"] == -(-M // 128) and pl["n_tiles"] == -(-N // pl["tile_n"])
             assert pl["waves"] == -(-(pl["m_tiles"] * pl["n_tiles"]) // 148)
     assert binding.plan_gemm(12544, 64, 256)["b_resident"] == 1 and binding.plan_gemm(8192, 8192, 8192)["b_resident"] == 0
-    assert binding.plan_gemm(8192, 8192, 8192)["tile_n"] == 256
+    big = binding.plan_gemm(8192, 8192, 8192)
+    # the large square GEMMs run on CTA pairs: 256 x 256 tiles, six ring slots, one worker per pair of SMs
+    assert (big["tile_m"], big["tile_n"], big["cta_group"], big["stages"], big["workers"]) == (256, 256, 2, 6, 74)
+    assert big["m_tiles"] == 32 and big["n_tiles"] == 32 and big["waves"] == -(-1024 // 74) and big["raster_group"] == 16
+    small = binding.plan_gemm(256, 256, 256)
+    assert small["cta_group"] == 1 and small["tile_m"] == 128 and small["workers"] == small["m_tiles"] * small["n_tiles"]
+    skinny = binding.plan_gemm(262144, 64, 256)
+    assert (skinny["tile_n"], skinny["cta_group"], skinny["stages"], skinny["b_resident"], skinny["workers"]) == (64, 1, 6, 1, 148)
+    sticky = binding.plan_gemm(3136, 2048, 512)         # short K, several tiles per worker: column-sticky order
+    assert sticky["sticky"] == 1 and sticky["tile_n"] == 128
     try:
         base = binding.plan_gemm(1024, 1024, 1024)["tile_n"]
         other = 128 if base != 128 else 64
@@ -123,4 +132,21 @@ def test_tile_plan_and_class_reuse(L):
             binding.set_class_tile(c, 0)
     assert binding.plan_gemm(1024, 1024, 1024)["tile_n"] == base
     assert L.i8ops_set_class_tile(3, 64) == 5 and L.i8ops_set_class_tile(0, 100) == 5
+    # a full class entry: (tile, cta_group, raster group, sticky) found on a base shape is reused by shapes within a
+    # factor of four of it, and by no others
+    try:
+        binding.set_class_plan(0, base=(1024, 1024, 1024), tile_n=128, cta_group=1, raster_group=4, sticky=0)
+        for (M, N, K) in table[0]:
+            pl = binding.plan_gemm(M, N, K)
+            assert (pl["tile_n"], pl["cta_group"], pl["raster_group"], pl["sticky"]) == (128, 1, 4, 0)
+        far = binding.plan_gemm(8192, 8192, 8192)
+        assert (far["tile_n"], far["cta_group"], far["raster_group"]) == (256, 2, 16)      # too far from the base: the rule decides
+        binding.set_class_plan(0, base=(4096, 4096, 4096), cta_group=1, tile_n=256)
+        assert binding.plan_gemm(4096, 4096, 4096)["cta_group"] == 1 and binding.plan_gemm(4096, 4096, 4096)["tile_m"] == 128
+    finally:
+        binding.set_class_plan(0, base=(8192, 8192, 8192), tile_n=256, cta_group=2, raster_group=16)    # the seeded entries
+        binding.set_class_plan(1, base=(262144, 64, 256), tile_n=64, cta_group=1, raster_group=16)
+    assert L.i8ops_set_class_plan(0, 1024, 0, 1024, 128, 0, 0, -1) == 5      # a base shape is all three extents or none
+    assert L.i8ops_set_class_plan(0, 0, 0, 0, 128, 2, 0, -1) == 5            # CTA pairs imply 256-wide tiles
+    assert L.i8ops_set_class_plan(0, 0, 0, 0, 0, 3, 0, -1) == 5 and L.i8ops_set_class_plan(0, 0, 0, 0, 0, 0, 65, -1) == 5
     assert L.i8ops_plan_gemm(0, 1, 1, 148, None) == 1

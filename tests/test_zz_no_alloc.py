@@ -4,7 +4,8 @@
 Its device copies live in a fixed 16 MiB array inside the library instead of a cudaMalloc'ed workspace.  The file is
 named so that pytest collects it after every other test: a run that stops at the first failure has then already run
 the rest.  The GPU test calls the C ABI twice in a row with different shapes, so the second call finds the array
-full of the first call's data, and compares each result bit for bit with what gemm_i8_host returns."""
+full of the first call's data, and compares each result bit for bit with what gemm_i8_host returns and with the CPU
+oracle."""
 import numpy as np
 import pytest
 
@@ -39,6 +40,7 @@ def test_rejects_problems_beyond_the_fixed_workspace():
 
 @pytest.mark.gpu
 def test_matches_gemm_i8_host_on_two_calls_in_a_row():
+    import oracle
     import paper_2505_18574_b200 as i8
     # a large problem first (tensor path, fills most of the array), then a smaller ragged one whose regions start
     # at other offsets and without a bias, then the first again
@@ -51,5 +53,7 @@ def test_matches_gemm_i8_host_on_two_calls_in_a_row():
         got = np.full((M, N), 0x33, np.int8)
         i8.gemm_i8_host_noalloc(p.A, p.B, got, bias, p.mult, p.shift, 1, 1)
         assert np.array_equal(got, want), f"call {i}: {M}x{N}x{K} differs from gemm_i8_host"
+        ref = oracle.gemm_i8(p.A, K, 1, p.B, 1, K, N, bias, p.mult, p.shift, 1, M, N, K, 1)
+        assert np.array_equal(got, ref), f"call {i}: {M}x{N}x{K} differs from the oracle"
         assert len(np.unique(want)) > 16, "degenerate output would prove nothing"
     assert i8.last_device_status() == 0
