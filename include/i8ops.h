@@ -64,7 +64,10 @@ typedef enum {
     I8_PATH_TENSOR = 2,     /* TMA -> shared memory ring -> tcgen05.mma kind::i8 -> tensor memory -> epilogue */
     I8_PATH_SMALL = 3,      /* small-tile tensor path: paired 64x64 problems */
     I8_PATH_TENSOR_2SM = 4, /* tensor path on clusters of two CTAs (tcgen05.mma.cta_group::2, 256 x 256 tiles) */
-    I8_PATH_CONV_SLAB = 5   /* stride-1 convolution with the input slab resident in shared memory and reused across taps */
+    I8_PATH_CONV_SLAB = 5,  /* stride-1 convolution with the input slab resident in shared memory and reused across taps */
+    I8_PATH_CHANNEL_MAJOR = 6,     /* tensor path computing the transposed product: 128 output channels on the tensor-memory
+                                      lanes, a strip of output rows on the columns (strip width chosen per problem) */
+    I8_PATH_CHANNEL_MAJOR_2SM = 7  /* the same on clusters of two CTAs: 256 output channels per tile */
 } i8_path;
 
 /*
@@ -264,7 +267,8 @@ int i8ops_last_path(void);
 
 /* Restrict dispatch: 0 = automatic (default), 1 = always the generic kernel, 2 = GEMMs and convolutions take the
  * two-SM tensor kernel whenever the layout allows the tensor path (also where its large tiles do not pay),
- * 3 = automatic, but stride-1 convolutions stay on the implicit-GEMM kernel instead of the slab kernel.
+ * 3 = automatic, but stride-1 convolutions stay on the implicit-GEMM kernel instead of the slab kernel,
+ * 4 = GEMMs and implicit-GEMM convolutions take the channel-major kernel whenever the layout allows the tensor path.
  * Returns the previous setting. */
 int i8ops_set_path(int mode);
 

@@ -15,6 +15,7 @@ _LIB_PATH = os.path.join(_HERE, "libi8ops.so")
 _lib = None
 
 PATH_NONE, PATH_GENERIC, PATH_TENSOR, PATH_SMALL, PATH_TENSOR_2SM, PATH_CONV_SLAB = 0, 1, 2, 3, 4, 5
+PATH_CHANNEL_MAJOR, PATH_CHANNEL_MAJOR_2SM = 6, 7
 
 _vp = ctypes.c_void_p
 _i64 = ctypes.c_int64

@@ -13,6 +13,7 @@
 #include "../../include/i8ops.h"
 #include "batched_tc.cuh"
 #include "conv_slab.cuh"
+#include "gemm_swap.cuh"
 #include "gemm_tc.cuh"
 #include "generic.cuh"
 #include "mpc.cuh"
@@ -48,11 +49,15 @@ static int g_force_bn = -1;                      // tuning override from the env
 static int g_tma_store = 1;                      // read-out of the wide tiles through TMA stores (I8OPS_TMA_STORE=0 turns it off)
 static int g_sticky = 1;                         // column-sticky tile order for short-K problems (I8OPS_STICKY=0 turns it off)
 static int g_tmap_cache = 1;                     // per-thread cache of encoded tensor maps (I8OPS_TMAP_CACHE=0 encodes every time)
+static int g_swap = 0;                           // channel-major kernel: 0 never, 1 by rule, 2 wherever legal (I8OPS_SWAP)
+static int g_swap_stages = 0;                    // ring slots of the channel-major kernel: 0 = as many as fit (I8OPS_SWAP_STAGES)
+static int g_swap_pw = 0;                        // strip width override for tuning (I8OPS_SWAP_PW)
 static int g_slab = 1;                           // slab-resident stride-1 convolution kernel (I8OPS_SLAB=0 turns it off)
 
 static thread_local int t_last_path = I8_PATH_NONE;
 static thread_local int t_last_cuda = 0;
 static thread_local bool t_used_two_sm = false;
+static thread_local bool t_used_swap = false;     // the last tensor-path launch was the channel-major kernel
 static thread_local bool t_tmap_failed = false;   // the last tensor-path attempt stopped at a tensor-map encoding (nothing launched)
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -64,6 +69,11 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                    CUtensorMapFloatOOBfill);
 static EncodeIm2colFn g_encode_im2col = nullptr;
+
+static int tensor_path_used() {
+    if (t_used_swap) return t_used_two_sm ? I8_PATH_CHANNEL_MAJOR_2SM : I8_PATH_CHANNEL_MAJOR;
+    return t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
+}
 
 static int cuda_fail(cudaError_t e) {
     t_last_cuda = (int)e;
@@ -110,6 +120,12 @@ static int get_ctx(DeviceCtx** out) {
         if (sticky) g_sticky = atoi(sticky);
         const char* slab = getenv("I8OPS_SLAB");
         if (slab) g_slab = atoi(slab);
+        const char* sw = getenv("I8OPS_SWAP");
+        if (sw) g_swap = atoi(sw);
+        const char* sws = getenv("I8OPS_SWAP_STAGES");
+        if (sws) g_swap_stages = atoi(sws);
+        const char* swp = getenv("I8OPS_SWAP_PW");
+        if (swp) g_swap_pw = atoi(swp);
         const char* tmc = getenv("I8OPS_TMAP_CACHE");
         if (tmc) g_tmap_cache = atoi(tmc);
         const char* pdl = getenv("I8OPS_PDL");
@@ -411,7 +427,15 @@ static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap
     t_last_plan = pl;
     t_used_two_sm = two_sm;
     CUtensorMap tmB;
-    {
+    if (kl.b_mn) {
+        // B stored with N contiguous: K rows of 128 (64-wide tiles: 64) bytes of N
+        const uint32_t mnw = b_rows >= 128 ? 128u : 64u;
+        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)K};
+        const uint64_t str[1] = {(uint64_t)ldb};
+        const uint32_t box[2] = {mnw, (uint32_t)BK};
+        int rc = make_tmap(&tmB, B, 2, dims, str, box, mnw == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
+        if (rc) return rc;
+    } else {
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
         const uint64_t str[1] = {(uint64_t)ldb};
         const uint32_t box[2] = {(uint32_t)kl.cb, (uint32_t)b_rows};
@@ -453,7 +477,7 @@ static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap
         p.sched.inv_cb1 = pl.sticky ? inv32(pl.col_base + 1) : 0xffffffffu;
     }
     p.kl = kl;
-    p.kl.b_resident = pl.b_resident;
+    p.kl.b_resident = kl.b_mn ? 0 : pl.b_resident;            // the resident-B fetch is written for K-major B only
     p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);   // SM clock stays below 2 GHz: at least the asked time
     p.dev_status = ctx->dev_status;
     if (two_sm) {
@@ -480,6 +504,11 @@ static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap
     }
 }
 
+static int run_gemm_swap(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
+                         const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N, int K,
+                         int relu, cudaStream_t st);
+static bool swap_wanted(int M, int N, int num_kb, int sm_count);
+
 static KLoop gemm_kloop(int K) {
     KLoop kl{};
     kl.cb = BK; kl.nsub = 1; kl.num_kblocks = (K + BK - 1) / BK;
@@ -488,18 +517,145 @@ static KLoop gemm_kloop(int K) {
     return kl;
 }
 
+// a_mn / b_mn: the operand is stored with M (A) or N (B) contiguous instead of K; lda / ldb is then the stride between K rows.
 static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                        const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N,
-                       int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
-    const KLoop kl = gemm_kloop(K);
+                       int K, int relu, cudaStream_t st, const RawOut& raw = RawOut(), int a_mn = 0, int b_mn = 0) {
+    KLoop kl = gemm_kloop(K);
+    kl.a_mn = a_mn; kl.b_mn = b_mn;
+    t_used_swap = false;
+    if (!raw.D && !a_mn && !b_mn && swap_wanted(M, N, kl.num_kblocks, ctx->sm_count)) {
+        int rc = run_gemm_swap(ctx, A, lda, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
+        if (rc != I8_ERR_UNSUPPORTED) { t_used_swap = rc == I8_OK; return rc; }
+    }
     const TcPlan pl = plan_tc(false, M, N, K, kl.num_kblocks, kl.num_iters, kl.num_kblocks, BK, ctx->sm_count);
     CUtensorMap tmA;
-    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
+    const uint64_t dims_k[2] = {(uint64_t)K, (uint64_t)M}, dims_m[2] = {(uint64_t)M, (uint64_t)K};
     const uint64_t str[1] = {(uint64_t)lda};
-    const uint32_t box[2] = {BK, BM};
-    int rc = make_tmap(&tmA, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+    const uint32_t box[2] = {BK, BM};                  // K-major: 128 bytes of K x 128 rows; MN-major: 128 rows x 128 of K
+    int rc = make_tmap(&tmA, A, 2, a_mn ? dims_m : dims_k, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
     return run_tc(ctx, false, pl, tmA, kl, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
+}
+
+// ------------------------------------------------------------------------------------------------ channel-major kernel
+// Plan of one launch of gemm_i8_swap_kernel: strip width, ring depth, shared-memory layout.
+struct SwapPlan {
+    int two_sm, pw, b_rows, stages, workers, m_tiles, n_blocks, num_tiles, tmem_cols;
+    int off_b, off_bar, smem_bytes;
+    double cycles;             // the cost model's estimate for the whole launch
+};
+
+// Strip width: every candidate (multiples of 16) is priced as waves x (ring slots per tile x cycles per slot + a fixed
+// cost per tile) + the exposed read-out of the last tile.  A slot's cycles are the larger of its four instructions
+// (pw / 2 cycles each, at least 48: narrower instructions are bound by operand reads) and its operand bytes at the
+// ~80 bytes per clock an SM draws from L2.
+static SwapPlan plan_swap(int M, int N, int num_iters, bool two_sm, int sm_count) {
+    SwapPlan best = {};
+    best.cycles = 1e300;
+    const int tile_ch = two_sm ? 256 : 128;
+    const int n_blocks = (N + tile_ch - 1) / tile_ch;
+    const int max_workers = two_sm ? sm_count / 2 : sm_count;
+    for (int pw = 256; pw >= 16; pw -= 16) {
+        if (g_swap_pw && pw != g_swap_pw) continue;
+        const int m_tiles = (M + pw - 1) / pw;
+        const int64_t tiles = (int64_t)m_tiles * n_blocks;
+        if (tiles >= (1ll << 30)) continue;
+        const int64_t waves = (tiles + max_workers - 1) / max_workers;
+        const int b_rows = two_sm ? pw / 2 : pw;
+        const double mma = 4.0 * (pw / 2 > 48 ? pw / 2 : 48);
+        const double feed = (16384.0 + 128.0 * b_rows) / 80.0;
+        const double cyc = (double)waves * ((double)num_iters * (mma > feed ? mma : feed) + 500.0) + 4.0 * pw;
+        if (cyc < best.cycles - 1e-9) {
+            best.cycles = cyc; best.pw = pw; best.b_rows = b_rows; best.m_tiles = m_tiles; best.n_blocks = n_blocks;
+            best.num_tiles = (int)tiles; best.workers = (int)(tiles < max_workers ? tiles : max_workers);
+        }
+    }
+    best.two_sm = two_sm ? 1 : 0;
+    if (!best.pw) return best;
+    int cols = 32;
+    while (cols < 2 * best.pw) cols *= 2;
+    best.tmem_cols = cols;
+    const int b_stage = best.b_rows * 128;
+    const int stage_bytes = 16384 + b_stage;
+    const int fixed = (2 * SWAP_MAX_STAGES + 4) * 8 + 16;
+    int stages = (226 * 1024 - fixed) / stage_bytes;
+    if (stages > SWAP_MAX_STAGES) stages = SWAP_MAX_STAGES;
+    if (g_swap_stages >= 2 && g_swap_stages < stages) stages = g_swap_stages;
+    stages &= ~1;                                        // two producers alternate ring slots
+    best.stages = stages;
+    best.off_b = stages * 16384;
+    best.off_bar = best.off_b + stages * b_stage;
+    best.smem_bytes = best.off_bar + fixed + 1024;
+    return best;
+}
+
+template <bool CONV, bool TWO_SM>
+static int launch_swap(DeviceCtx* ctx, int slot, const SwapPlan& pl, const CUtensorMap& tmW, const CUtensorMap& tmX, const SwapParams& p,
+                       cudaStream_t st) {
+    auto kern = gemm_i8_swap_kernel<CONV, TWO_SM>;
+    if (!ctx->attr_set[slot]) {
+        CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        ctx->attr_set[slot] = true;
+    }
+    CUDA_TRY(launch_kernel(kern, true, TWO_SM ? 2 : 1, TWO_SM ? 2 * pl.workers : pl.workers, 32 * (CONV ? 3 : 2) + 32 * SWAP_EPI_WARPS,
+                           (size_t)pl.smem_bytes, st, tmW, tmX, p));
+    return I8_OK;
+}
+
+// W: [N][ldw] K-contiguous weights (the caller's B); tmX: the map of the other operand, built by the caller for the
+// plan's b_rows.  C row-major [M][ldc].
+static int run_swap(DeviceCtx* ctx, bool conv, const SwapPlan& pl, const CUtensorMap& tmX, const KLoop& kl, const int8_t* W, int64_t ldw,
+                    int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
+                    int M, int N, int K, int relu, cudaStream_t st) {
+    CUtensorMap tmW;
+    {
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
+        const uint64_t str[1] = {(uint64_t)ldw};
+        const uint32_t box[2] = {(uint32_t)kl.cb, (uint32_t)BM};
+        int rc = make_tmap(&tmW, W, 2, dims, str, box, swizzle_for(kl.cb));
+        if (rc) return rc;
+    }
+    SwapParams p;
+    p.C = C; p.ldc = ldc; p.bias = bias; p.mult = mult; p.shift = shift; p.per_channel = per_channel; p.relu = relu;
+    p.M = M; p.N = N; p.K = K;
+    p.pw = pl.pw; p.b_rows = pl.b_rows;
+    p.c_word_ok = ((reinterpret_cast<uintptr_t>(C) & 3u) == 0 && ldc % 4 == 0 && N % 4 == 0) ? 1 : 0;
+    p.m_tiles = pl.m_tiles; p.n_blocks = pl.n_blocks; p.num_tiles = pl.num_tiles;
+    p.inv_nb = pl.n_blocks <= 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)pl.n_blocks);
+    p.stages = pl.stages; p.b_stage_bytes = pl.b_rows * 128; p.tmem_cols = pl.tmem_cols;
+    p.off_b = pl.off_b; p.off_bar = pl.off_bar;
+    p.kl = kl;
+    p.kl.b_resident = 0;
+    p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);
+    p.dev_status = ctx->dev_status;
+    t_used_two_sm = pl.two_sm != 0;
+    if (conv) return pl.two_sm ? launch_swap<true, true>(ctx, 21, pl, tmW, tmX, p, st) : launch_swap<true, false>(ctx, 22, pl, tmW, tmX, p, st);
+    return pl.two_sm ? launch_swap<false, true>(ctx, 23, pl, tmW, tmX, p, st) : launch_swap<false, false>(ctx, 24, pl, tmW, tmX, p, st);
+}
+
+// Whether a problem goes to the channel-major kernel.  Forced (path mode 4, I8OPS_SWAP=2): whenever it is legal.  By
+// rule: problems too small for the 256 x 256 pair kernel to pay, with at least 128 output channels.
+static bool swap_wanted(int M, int N, int num_kb, int sm_count) {
+    if (g_path_mode == 4 || g_swap == 2) return true;
+    if (!g_swap || g_path_mode != 0 || g_force_bn >= 0) return false;
+    if (N < 128) return false;
+    return !(g_tc2 && pair_pays(M, N, 256, num_kb, sm_count));
+}
+
+static int run_gemm_swap(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
+                         const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N, int K,
+                         int relu, cudaStream_t st) {
+    const KLoop kl = gemm_kloop(K);
+    const SwapPlan pl = plan_swap(M, N, kl.num_iters, N > 128, ctx->sm_count);
+    if (!pl.pw || pl.stages < 2) return I8_ERR_UNSUPPORTED;
+    CUtensorMap tmX;
+    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
+    const uint64_t str[1] = {(uint64_t)lda};
+    const uint32_t box[2] = {BK, (uint32_t)pl.b_rows};
+    int rc = make_tmap(&tmX, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    return run_swap(ctx, false, pl, tmX, kl, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
 }
 
 // Implicit-GEMM convolution: A tiles come from an im2col-mode tensor map over the NHWC activations.
@@ -508,11 +664,6 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
                        int stride_h, int stride_w, int pad_h, int pad_w, int relu, cudaStream_t st) {
     const int cb = C % 128 == 0 ? 128 : (C % 64 == 0 ? 64 : 32);
     const int M = N * P * Q;
-    CUtensorMap tmA;
-    {
-        int rc = make_tmap_im2col(&tmA, x, N, H, W, C, R, S, stride_h, stride_w, pad_h, pad_w, cb, BM, swizzle_for(cb));
-        if (rc) return rc;
-    }
     KLoop kl{};
     kl.cb = cb; kl.nsub = BK / cb; kl.cblocks = C / cb; kl.num_kblocks = R * S * kl.cblocks;
     kl.P = P; kl.Q = Q; kl.S = S;
@@ -522,6 +673,23 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     kl.mmas_last = (kl.num_kblocks - (kl.num_iters - 1) * kl.nsub) * (cb / 32);
     kl.stride_h = stride_h; kl.stride_w = stride_w; kl.pad_h = pad_h; kl.pad_w = pad_w;
     const int K = R * S * C;
+    t_used_swap = false;
+    if (swap_wanted(M, Kf, (K + BK - 1) / BK, ctx->sm_count)) {
+        // filters on the tensor-memory lanes, a strip of output pixels on the columns
+        const SwapPlan sp = plan_swap(M, Kf, kl.num_iters, Kf > 128, ctx->sm_count);
+        if (sp.pw && sp.stages >= 2) {
+            CUtensorMap tmX;
+            int rc = make_tmap_im2col(&tmX, x, N, H, W, C, R, S, stride_h, stride_w, pad_h, pad_w, cb, sp.b_rows, swizzle_for(cb));
+            if (rc) return rc;
+            t_used_swap = true;
+            return run_swap(ctx, true, sp, tmX, kl, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
+        }
+    }
+    CUtensorMap tmA;
+    {
+        int rc = make_tmap_im2col(&tmA, x, N, H, W, C, R, S, stride_h, stride_w, pad_h, pad_w, cb, BM, swizzle_for(cb));
+        if (rc) return rc;
+    }
     // CTA pairs for convolutions follow the same measured rule as for GEMMs, or are asked for explicitly (path mode 2, I8OPS_CONV2SM=1)
     const TcPlan pl = plan_tc(true, M, Kf, K, (K + BK - 1) / BK, kl.num_iters, kl.num_kblocks, cb, ctx->sm_count);
     return run_tc(ctx, true, pl, tmA, kl, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
@@ -680,12 +848,15 @@ int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_
     rc = get_ctx(&ctx);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    const bool tc_legal = K >= 1 && a_cs == 1 && b_rs == 1 && aligned16(A) && aligned16(B) && a_rs % 16 == 0 &&
-                          b_cs % 16 == 0 && a_rs >= K && b_cs >= K;
+    // the tensor path takes either storage order of either operand: K contiguous (K-major) or M / N contiguous
+    const bool a_k = a_cs == 1 && a_rs % 16 == 0 && a_rs >= K, a_m = !a_k && a_rs == 1 && a_cs % 16 == 0 && a_cs >= M;
+    const bool b_k = b_rs == 1 && b_cs % 16 == 0 && b_cs >= K, b_n = !b_k && b_cs == 1 && b_rs % 16 == 0 && b_rs >= N;
+    const bool tc_legal = K >= 1 && aligned16(A) && aligned16(B) && (a_k || a_m) && (b_k || b_n);
     if (tc_legal && g_path_mode != 1) {
         t_used_two_sm = false; t_tmap_failed = false;
-        rc = run_gemm_tc(ctx, A, a_rs, B, b_cs, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
-        if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
+        rc = run_gemm_tc(ctx, A, a_k ? a_rs : a_cs, B, b_k ? b_cs : b_rs, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, RawOut(),
+                         a_m ? 1 : 0, b_n ? 1 : 0);
+        if (rc == I8_OK) t_last_path = tensor_path_used();
         if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         // the driver refused a tensor map for this geometry: nothing was launched, the generic kernel serves it
     }
@@ -707,13 +878,16 @@ int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, in
     int rc = get_ctx(&ctx);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    const bool tc_legal = K >= 1 && a_cs == 1 && b_rs == 1 && aligned16(A) && aligned16(B) && a_rs % 16 == 0 &&
-                          b_cs % 16 == 0 && a_rs >= K && b_cs >= K;
+    // the tensor path takes either storage order of either operand: K contiguous (K-major) or M / N contiguous
+    const bool a_k = a_cs == 1 && a_rs % 16 == 0 && a_rs >= K, a_m = !a_k && a_rs == 1 && a_cs % 16 == 0 && a_cs >= M;
+    const bool b_k = b_rs == 1 && b_cs % 16 == 0 && b_cs >= K, b_n = !b_k && b_cs == 1 && b_rs % 16 == 0 && b_rs >= N;
+    const bool tc_legal = K >= 1 && aligned16(A) && aligned16(B) && (a_k || a_m) && (b_k || b_n);
     if (tc_legal && g_path_mode != 1) {
         RawOut raw; raw.D = D; raw.ldd = ldd; raw.accumulate = accumulate ? 1 : 0;
         t_used_two_sm = false; t_tmap_failed = false;
-        rc = run_gemm_tc(ctx, A, a_rs, B, b_cs, nullptr, 0, nullptr, nullptr, nullptr, 0, M, N, K, 0, st, raw);
-        if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
+        rc = run_gemm_tc(ctx, A, a_k ? a_rs : a_cs, B, b_k ? b_cs : b_rs, nullptr, 0, nullptr, nullptr, nullptr, 0, M, N, K, 0, st, raw,
+                         a_m ? 1 : 0, b_n ? 1 : 0);
+        if (rc == I8_OK) t_last_path = tensor_path_used();
         if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
     }
     GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, nullptr, 0, 0, nullptr, 0, nullptr, nullptr, 0, 0, 1, M, N, K,
@@ -778,7 +952,7 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
             // a 1x1 convolution is the GEMM [N*H*W, C] x [C, K]
             t_used_two_sm = false; t_tmap_failed = false;
             rc = run_gemm_tc(ctx, x, C, w, C, y, K, bias, mult, shift, per_channel, N * H * W, K, C, relu, st);
-            if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
+            if (rc == I8_OK) t_last_path = tensor_path_used();
             if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
         if (g_slab && g_path_mode == 0 && stride_h == 1 && stride_w == 1 && (int64_t)N * P * Q < (1ll << 31)) {
@@ -796,7 +970,7 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
             t_used_two_sm = false; t_tmap_failed = false;
             rc = run_conv_tc(ctx, x, w, y, bias, mult, shift, per_channel, N, H, W, C, K, R, S, P, Q, stride_h, stride_w,
                              pad_h, pad_w, relu, st);
-            if (rc == I8_OK) t_last_path = t_used_two_sm ? I8_PATH_TENSOR_2SM : I8_PATH_TENSOR;
+            if (rc == I8_OK) t_last_path = tensor_path_used();
             if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
     }
@@ -1048,7 +1222,7 @@ int i8ops_last_path(void) { return t_last_path; }
 
 int i8ops_set_path(int mode) {
     const int prev = g_path_mode;
-    if (mode >= 0 && mode <= 3) g_path_mode = mode;
+    if (mode >= 0 && mode <= 4) g_path_mode = mode;
     return prev;
 }
 

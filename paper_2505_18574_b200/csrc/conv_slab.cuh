@@ -285,6 +285,16 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         }
         const bool shift32 = named_barrier_and(2, EPI_THREADS, all32);
         const bool fold = named_barrier_and(3, EPI_THREADS, allfold);
+        // 64-filter tiles: a warp serves the same 32 filters for the whole kernel, so their constants live in registers.
+        // (Fetched from shared memory per output they cost the load/store pipe three wavefronts per column and warp, on the
+        // pipe that also delivers the tensor core's operands: the 64-wide instruction then issued every ~75 cycles
+        // instead of the ~48 its operand reads need.)
+        constexpr bool ONE_CHUNK = COLS_PER_GROUP == 32;
+        int32_t rm[ONE_CHUNK ? 32 : 1], rb[ONE_CHUNK ? 32 : 1];
+        if constexpr (ONE_CHUNK) if (fold) {
+#pragma unroll
+            for (int j = 0; j < 32; j++) { rm[j] = s_m2[cgroup * 32 + j]; rb[j] = s_bias[cgroup * 32 + j]; }
+        }
         // position of this thread's accumulator row in the tile's raster: (dy, dx) = (j / Wp, j % Wp)
         const int j = quarter * 32 + lane;
         const int dy = fast_div(j, p.Wp, p.inv_wp), dx = j - dy * p.Wp;
@@ -312,8 +322,13 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                 tmem_ld_wait();
                 uint32_t out[8];
                 if (fold) {
-                    if (p.relu) epilogue_chunk_fold<true>(v, s_m2, s_c64, c0, out);
-                    else epilogue_chunk_fold<false>(v, s_m2, s_c64, c0, out);
+                    if constexpr (ONE_CHUNK) {
+                        if (p.relu) epilogue_chunk_fold_add_regs<true>(v, rb, rm, out);
+                        else epilogue_chunk_fold_add_regs<false>(v, rb, rm, out);
+                    } else {
+                        if (p.relu) epilogue_chunk_fold<true>(v, s_m2, s_c64, c0, out);
+                        else epilogue_chunk_fold<false>(v, s_m2, s_c64, c0, out);
+                    }
                 } else if (shift32) {
                     if (p.relu) epilogue_chunk_shift32<true>(v, s_bias, s_m2, c0, out);
                     else epilogue_chunk_shift32<false>(v, s_bias, s_m2, c0, out);

@@ -42,6 +42,10 @@ struct KLoop {
     int stride_h, stride_w, pad_h, pad_w;
     uint32_t inv_pq, inv_q;               // floor(2^32 / (P*Q)) and floor(2^32 / Q) (0xffffffff for a divisor of 1)
     int b_resident;                       // the whole B operand of the (single) block column stays in shared memory
+    // GEMM only: an operand stored with its M (A) or N (B) extent contiguous is fetched as K rows of 128 (64 for 64-wide
+    // B tiles) contiguous bytes and consumed through an MN-major shared-memory descriptor: no transpose pass.  The maps
+    // then have the contiguous extent as dimension 0 and K as dimension 1.
+    int a_mn, b_mn;
 };
 
 // n / d for n < 2^31 with inv = floor(2^32 / d): the estimate is at most one too small.
@@ -196,6 +200,18 @@ __device__ __forceinline__ void epilogue_chunk_fold_regs(const int32_t (&v)[32],
     for (int j = 0; j < 8; j++) {
         const uint32_t pk = pack_sat4(requant_fold(v[4 * j + 0], rm[4 * j + 0], rc[4 * j + 0]), requant_fold(v[4 * j + 1], rm[4 * j + 1], rc[4 * j + 1]),
                                       requant_fold(v[4 * j + 2], rm[4 * j + 2], rc[4 * j + 2]), requant_fold(v[4 * j + 3], rm[4 * j + 3], rc[4 * j + 3]));
+        out[j] = RELU ? relu_s8x4(pk) : pk;
+    }
+}
+
+// Folded form, bias added explicitly, constants in registers (two words per channel).
+template <bool RELU>
+__device__ __forceinline__ void epilogue_chunk_fold_add_regs(const int32_t (&v)[32], const int32_t (&rb)[32], const int32_t (&rm)[32],
+                                                             uint32_t (&out)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+        const uint32_t pk = pack_sat4(requant_fold(v[4 * j + 0] + rb[4 * j + 0], rm[4 * j + 0], 1ll << 31), requant_fold(v[4 * j + 1] + rb[4 * j + 1], rm[4 * j + 1], 1ll << 31),
+                                      requant_fold(v[4 * j + 2] + rb[4 * j + 2], rm[4 * j + 2], 1ll << 31), requant_fold(v[4 * j + 3] + rb[4 * j + 3], rm[4 * j + 3], 1ll << 31));
         out[j] = RELU ? relu_s8x4(pk) : pk;
     }
 }
@@ -401,12 +417,24 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                         }
                         if (++c_idx == kl.cblocks) { c_idx = 0; if (++fs == kl.S) { fs = 0; ++fr; } }
                     } else if (leader) {
-                        if (TWO_SM) tma_load_2d_pair(dstA, &tmA, full, kbi * BK, row_a);
-                        else tma_load_2d(dstA, &tmA, full, kbi * BK, row_a);
+                        // K-major: (k, row); MN-major: (row, k), the 128 K rows of the slot 128 bytes apart
+                        const int ax = kl.a_mn ? row_a : kbi * BK, ay = kl.a_mn ? kbi * BK : row_a;
+                        if (TWO_SM) tma_load_2d_pair(dstA, &tmA, full, ax, ay);
+                        else tma_load_2d(dstA, &tmA, full, ax, ay);
                     }
                     if (leader && !bres) {
-                        if (TWO_SM) tma_load_2d_pair(dstB, &tmB, full, kbi * kl.cb, row_b);
-                        else tma_load_2d(dstB, &tmB, full, kbi * kl.cb, row_b);
+                        if (!CONV && kl.b_mn) {
+                            // one box of K rows per 128 columns of the tile (a 64-wide tile: one box of 64-byte rows)
+                            constexpr int NBOX = B_ROWS > 128 ? B_ROWS / 128 : 1;
+#pragma unroll
+                            for (int h = 0; h < NBOX; h++) {
+                                if (TWO_SM) tma_load_2d_pair(dstB + h * (128 * BK), &tmB, full, row_b + h * 128, kbi * BK);
+                                else tma_load_2d(dstB + h * (128 * BK), &tmB, full, row_b + h * 128, kbi * BK);
+                            }
+                        } else {
+                            if (TWO_SM) tma_load_2d_pair(dstB, &tmB, full, kbi * kl.cb, row_b);
+                            else tma_load_2d(dstB, &tmB, full, kbi * kl.cb, row_b);
+                        }
                     }
                 }
                 issued |= 1u << stage;
@@ -427,11 +455,17 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (whole warp loops, one lane issues)
-        constexpr uint32_t idesc = make_idesc_i8(TILE_M, BN, 0, 0);   // a pair's instruction spans both CTAs' rows
+        const uint32_t idesc = make_idesc_i8(TILE_M, BN, kl.a_mn, kl.b_mn);   // a pair's instruction spans both CTAs' rows
         // K-major operands: rows cb bytes apart, swizzled over cb bytes, 8-row groups 8*cb bytes apart;
         // a 32-byte step along K inside a swizzle row is a plain address offset.
         const uint64_t swz = kl.cb == 128 ? SWZ_128B : (kl.cb == 64 ? SWZ_64B : SWZ_32B);
-        const uint64_t desc_hi = make_smem_desc(0, 16, 8 * kl.cb, swz);   // everything but the start address
+        const uint64_t desc_k = make_smem_desc(0, 16, 8 * kl.cb, swz);   // everything but the start address
+        // MN-major operands: K rows of `mnw` contiguous bytes (128; 64 for a 64-wide B tile), swizzled over mnw bytes;
+        // 8 K rows are one group (stride offset 8 * mnw), the next block of mnw columns starts one whole box further
+        // (leading offset 128 rows * mnw), and 32 of K is 32 rows.
+        constexpr int B_MNW = B_ROWS >= 128 ? 128 : 64;
+        const uint64_t desc_hi_a = kl.a_mn ? make_smem_desc(0, 128 * 128, 8 * 128, SWZ_128B) : desc_k;
+        const uint64_t desc_hi_b = (!CONV && kl.b_mn) ? make_smem_desc(0, 128 * B_MNW, 8 * B_MNW, B_MNW == 128 ? SWZ_128B : SWZ_64B) : desc_k;
         const bool leader = elect_one();
         // A full ring slot always takes BK / 32 = 4 instructions; their operand offsets (in 16-byte descriptor
         // units) inside the slot depend only on the sub-block geometry.
@@ -440,8 +474,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
         for (int i = 0; i < 4; i++) {
             const int sub = i / per_sub, k = i - sub * per_sub;
-            offA[i] = (sub * a_sub_bytes + k * UMMA_K) >> 4;
-            offB[i] = (sub * b_sub_bytes + k * UMMA_K) >> 4;
+            offA[i] = (kl.a_mn ? i * UMMA_K * 128 : sub * a_sub_bytes + k * UMMA_K) >> 4;
+            offB[i] = ((!CONV && kl.b_mn) ? i * UMMA_K * B_MNW : sub * b_sub_bytes + k * UMMA_K) >> 4;
         }
         const uint32_t a_base = (sA & 0x3FFFFu) >> 4, b_base = (sB & 0x3FFFFu) >> 4;
         int stage = 0, ab = 0;
@@ -471,9 +505,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
                     for (int i = 0; i < 4; i++)
                         if (i < nm) {
-                            if (TWO_SM) mma_i8_ss_pair(d_tmem, desc_hi | (uint64_t)(a0 + offA[i]), desc_hi | (uint64_t)(b0 + offB[i]), idesc,
+                            if (TWO_SM) mma_i8_ss_pair(d_tmem, desc_hi_a | (uint64_t)(a0 + offA[i]), desc_hi_b | (uint64_t)(b0 + offB[i]), idesc,
                                                        (it | i) != 0 ? 1u : 0u);
-                            else mma_i8_ss(d_tmem, desc_hi | (uint64_t)(a0 + offA[i]), desc_hi | (uint64_t)(b0 + offB[i]), idesc,
+                            else mma_i8_ss(d_tmem, desc_hi_a | (uint64_t)(a0 + offA[i]), desc_hi_b | (uint64_t)(b0 + offB[i]), idesc,
                                            (it | i) != 0 ? 1u : 0u);
                         }
                     // slot reusable once these MMAs have read it (in a pair: in both CTAs)

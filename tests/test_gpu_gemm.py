@@ -78,9 +78,50 @@ def test_padded_leading_dimensions(M, N, K, pads):
 
 
 @pytest.mark.parametrize("a_layout,b_layout", [("row", "row"), ("col", "col"), ("col", "row")])
-def test_other_layouts_use_generic(a_layout, b_layout):
+def test_other_layouts_unaligned_use_generic(a_layout, b_layout):
+    """Leading dimensions that are not multiples of 16 bytes cannot be described to the copy engine."""
     p = inputs.make_gemm(70, 50, 90, 5, a_layout=a_layout, b_layout=b_layout, per_channel=1, relu=0, shift_lo=10, shift_hi=18)
     _both_paths(p, expect_tensor=False)
+
+
+@pytest.mark.parametrize("a_layout,b_layout", [("row", "row"), ("col", "col"), ("col", "row")])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (256, 64, 32), (300, 200, 100), (513, 96, 1040), (1000, 40, 48), (130, 130, 2048),
+                                   (384, 320, 16), (640, 1300, 144), (2048, 1536, 512), (77, 520, 272)])
+def test_mn_major_operands_on_the_tensor_path(a_layout, b_layout, M, N, K):
+    """Row-major B (the layout of the paper's printed GEMM listing, B[K][N]) and column-major A are consumed by the tensor
+    kernels through MN-major descriptors: every tile width, ragged edges, one CTA per tile and CTA pairs."""
+    import paper_2505_18574_b200 as i8
+    pa = (-(M if a_layout == "col" else K)) % 16
+    pb = (-(N if b_layout == "row" else K)) % 16
+    p = inputs.make_gemm(M, N, K, 8000 + M + N + K, a_layout=a_layout, b_layout=b_layout, per_channel=1, relu=M % 2,
+                         shift_lo=12, shift_hi=22, lda_pad=pa, ldb_pad=pb)
+    want = H.gemm_oracle(p)
+    for mode in (0, 2):
+        i8.set_path(mode)
+        got = H.gemm_gpu(p)
+        assert i8.last_path() == (i8.PATH_TENSOR_2SM if mode == 2 else i8.PATH_TENSOR), (mode, i8.last_path())
+        H.assert_same(got, want, f"{p.name} {a_layout}/{b_layout} mode {mode}")
+    i8.set_path(0)
+    assert i8.last_device_status() == 0
+
+
+def test_mn_major_closed_form():
+    """Oracle-independent: a one-hot A picks rows of a row-major B; with A stored column-major as well."""
+    import paper_2505_18574_b200 as i8
+    for a_layout in ("row", "col"):
+        p = inputs.make_gemm(128, 384, 128, 4, a_layout=a_layout, b_layout="row", per_channel=0, relu=0, with_bias=False)
+        p.A[:] = 0
+        for i in range(128):
+            k = (5 * i + 3) % 128
+            if a_layout == "row":
+                p.A[i, k] = 1
+            else:
+                p.A[k, i] = 1
+        p.mult[:] = 1; p.shift[:] = 0
+        got = H.gemm_gpu(p)
+        assert i8.last_path() in TENSOR_PATHS
+        want = np.stack([p.B[(5 * i + 3) % 128, :384] for i in range(128)])
+        assert np.array_equal(got, want), a_layout
 
 
 def test_unaligned_k_falls_back():
@@ -317,11 +358,11 @@ def test_tensor_map_cache_keys_on_the_address():
     h0, m0 = i8.tmap_cache_stats()
     H.assert_same(run(A1, B1), want, "first address again")
     h1, m1 = i8.tmap_cache_stats()
-    assert m1 == m0 and h1 >= h0 + 3, "the repeated call must reuse its three maps (A, B, C)"
+    assert m1 == m0 and h1 >= h0 + 2, "the repeated call must reuse its maps (A and B; C too where the read-out uses TMA stores)"
     A2.zero_()                                             # were the first address's map reused, the result would not change
     got = run(A2, B1)
     h2, m2 = i8.tmap_cache_stats()
-    assert m2 == m1 + 1 and h2 >= h1 + 2, "only A moved: one new map"
+    assert m2 == m1 + 1 and h2 >= h1 + 1, "only A moved: one new map"
     assert not np.array_equal(got, want)
     A2.copy_(A1)
     H.assert_same(run(A2, B2), want, "second address")
