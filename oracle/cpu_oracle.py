@@ -28,7 +28,7 @@ def build(force: bool = False) -> str:
     """Compile ``oracle.c`` into ``liboracle.so`` beside it (gcc, OpenMP over output rows)."""
     if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
         cmd = ["gcc", "-O3", "-march=native", "-fopenmp", "-fPIC", "-shared", "-std=c11",
-               "-Wall", "-Wextra", "-o", _SO, _SRC]
+               "-Wall", "-Wextra", "-o", _SO, _SRC, "-lm"]
         subprocess.run(cmd, check=True)
     return _SO
 
@@ -38,6 +38,11 @@ def _bind(path: str):
     L.oracle_requant.restype = ctypes.c_int32
     L.oracle_requant.argtypes = [_i64, ctypes.c_int32, _int, ctypes.c_int32, ctypes.c_int32,
                                  ctypes.POINTER(_int)]
+    L.oracle_requant_fscale.restype = ctypes.c_int32
+    L.oracle_requant_fscale.argtypes = [_i64, ctypes.c_int32, _int, ctypes.c_float, ctypes.POINTER(_int)]
+    L.oracle_gemm_i8_fscale.restype = _int
+    L.oracle_gemm_i8_fscale.argtypes = [_i8p, _i64, _i64, _i8p, _i64, _i64, _i8p, _i64, _i32p,
+                                        ctypes.POINTER(ctypes.c_float), _int, _int, _int, _int, _int]
     L.oracle_gemm_acc.restype = None
     L.oracle_gemm_acc.argtypes = [_i8p, _i64, _i64, _i8p, _i64, _i64, _i64p, _int, _int, _int]
     L.oracle_gemm_i8.restype = _int
@@ -84,6 +89,20 @@ class Oracle:
         ovf = _int(0)
         v = self._L.oracle_requant(int(acc), int(bias), int(relu), int(mult), int(shift), ctypes.byref(ovf))
         return int(v), int(ovf.value)
+
+    def requant_fscale(self, acc: int, bias: int, relu: int, scale: float):
+        """Return (int8 value, overflow flag) of one float-scale read-out (scale is taken as a binary32 value)."""
+        ovf = _int(0)
+        v = self._L.oracle_requant_fscale(int(acc), int(bias), int(relu), ctypes.c_float(scale), ctypes.byref(ovf))
+        return int(v), int(ovf.value)
+
+    def gemm_i8_fscale(self, A, a_rs, a_cs, B, b_rs, b_cs, ldc, bias, scale, per_channel, M, N, K, relu):
+        """C as an (M, ldc) int8 array; scale: float32 array of 1 or N entries."""
+        assert scale.dtype == np.float32 and scale.flags["C_CONTIGUOUS"]
+        C = np.zeros((M, ldc), dtype=np.int8)
+        self._L.oracle_gemm_i8_fscale(_p8(A), a_rs, a_cs, _p8(B), b_rs, b_cs, _p8(C), ldc, _p32(bias),
+                                      scale.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), per_channel, M, N, K, relu)
+        return C
 
     def gemm_acc(self, A, a_rs, a_cs, B, b_rs, b_cs, M, N, K) -> np.ndarray:
         acc = np.empty((M, N), dtype=np.int64)
@@ -164,6 +183,14 @@ def requant(*a, **k):
 
 def gemm_acc(*a, **k):
     return lib().gemm_acc(*a, **k)
+
+
+def requant_fscale(*a, **k):
+    return lib().requant_fscale(*a, **k)
+
+
+def gemm_i8_fscale(*a, **k):
+    return lib().gemm_i8_fscale(*a, **k)
 
 
 def gemm_i8(*a, **k):

@@ -36,11 +36,21 @@
  * pre-scale value (after the bias add) leaves the int32 range, which puts the case outside the
  * library's contract.
  *
+ * Float-scale read-out (oracle_requant_fscale, oracle_gemm_i8_fscale): the paper's Gemmini listings pass
+ * the read-out scale as a single-precision float (the store configuration of the ISA description, e.g. 1.0f in
+ * the printed GEMM).  The paper gives no rounding rule; the reading taken here is IEEE-754 binary32 arithmetic, the
+ * precision the paper fixes for that argument:
+ *     y   = fl32( fl32(t) * scale )      t = acc + bias after the optional ReLU, converted and multiplied with
+ *                                        round-to-nearest-even
+ *     out = min(127, max(-128, rne(y)))  rne = round to nearest integer, ties to even
+ * With scale = 1.0f this is again the saturating C = A*B of the printed listing.
+ *
  * Threads (OpenMP) split output rows only; every output element is still produced by the plain
  * loops below in k order.
  */
 #include <stdint.h>
 #include <stddef.h>
+#include <math.h>
 #ifdef _OPENMP
 #include <omp.h>
 #endif
@@ -66,6 +76,43 @@ int32_t oracle_requant(int64_t acc, int32_t bias, int relu, int32_t mult, int32_
     if (u > 127) u = 127;
     if (u < -128) u = -128;
     return (int32_t)u;
+}
+
+/* One float-scale read-out: bias -> ReLU -> binary32 multiply -> round to nearest even -> clamp to int8.
+ * (The default rounding mode is round-to-nearest-even; nothing in this library changes it.) */
+int32_t oracle_requant_fscale(int64_t acc, int32_t bias, int relu, float scale, int *overflow)
+{
+    int64_t t = acc + (int64_t)bias;
+    if (overflow && (t > (int64_t)INT32_MAX || t < (int64_t)INT32_MIN)) *overflow = 1;
+    if (relu && t < 0) t = 0;
+    volatile float tf = (float)(int32_t)t;      /* int32 -> binary32, one rounding */
+    volatile float y = tf * scale;              /* one binary32 multiplication, one rounding */
+    if (y != y) return 0;                       /* NaN scale: defined as 0 */
+    if (y >= 127.0f) return 127;
+    if (y <= -128.0f) return -128;
+    return (int32_t)lrintf(y);                  /* nearest integer, ties to even */
+}
+
+/* C[m*ldc+n] = float-scale read-out of sum_k A[..]*B[..]; scale has one entry or N entries. */
+int oracle_gemm_i8_fscale(const int8_t *A, int64_t a_rs, int64_t a_cs,
+                          const int8_t *B, int64_t b_rs, int64_t b_cs,
+                          int8_t *C, int64_t ldc,
+                          const int32_t *bias, const float *scale, int per_channel,
+                          int M, int N, int K, int relu)
+{
+    int overflow = 0;
+    #pragma omp parallel for schedule(static) reduction(|:overflow)
+    for (int m = 0; m < M; m++)
+        for (int n = 0; n < N; n++) {
+            int64_t acc = 0;
+            for (int k = 0; k < K; k++)
+                acc += (int32_t)A[m * a_rs + k * a_cs] * (int32_t)B[k * b_rs + n * b_cs];
+            int ovf = 0;
+            C[m * ldc + n] = (int8_t)oracle_requant_fscale(acc, bias ? bias[n] : 0, relu,
+                                                           scale[per_channel ? n : 0], &ovf);
+            overflow |= ovf;
+        }
+    return overflow;
 }
 
 /* Raw accumulators of a GEMM (no epilogue), for tests that pin the sum on its own. */

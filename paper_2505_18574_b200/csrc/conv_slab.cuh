@@ -116,8 +116,7 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         tma_prefetch_desc(&tmX);
         tma_prefetch_desc(&tmW);
     }
-    grid_launch_dependents();
-    grid_dependency_wait();          // global memory is touched from here on
+    grid_launch_dependents();        // the next kernel may be scheduled; this one waits for its predecessor after set-up
     // Set-up barrier.  The producer warp initialised the mbarriers itself and needs nothing from the others, so it only
     // signals and starts loading at once; everybody else waits for the barriers and the tensor-memory address.
     uint32_t tmem_base = 0;
@@ -133,6 +132,7 @@ conv_slab_i8_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 
     const int taps = p.R * p.S;
     const uint32_t w_sub_bytes = BN * p.cb;          // one (tap, channel block) of the filter bank
+    grid_dependency_wait();          // global memory is touched from here on
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer

@@ -27,7 +27,10 @@
 namespace i8 {
 
 constexpr int SWAP_MAX_STAGES = 8;
-constexpr int SWAP_EPI_WARPS = 8;
+#ifndef SWAP_EPI_WARPS_N
+#define SWAP_EPI_WARPS_N 8
+#endif
+constexpr int SWAP_EPI_WARPS = SWAP_EPI_WARPS_N;      // a multiple of 4: warps sharing a lane quarter split the strip's columns
 constexpr int SWAP_UNIT = 16;                         // granularity of the strip width (tcgen05.mma: N is a multiple of 16)
 
 struct SwapParams {
@@ -179,9 +182,9 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         tma_prefetch_desc(&tmW);
         tma_prefetch_desc(&tmX);
     }
-    // Everything above touched only shared and tensor memory; from here on global memory is read and written.
+    // The next kernel of the stream may be scheduled from here on; this one goes on with set-up that touches only shared
+    // and tensor memory, and waits for its own predecessor right before the roles start (below).
     grid_launch_dependents();
-    grid_dependency_wait();
     uint32_t tmem_base = 0;
     if (TWO_SM) {
         tc_fence_before();
@@ -207,6 +210,8 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     const uint32_t full0 = TWO_SM ? map_to_cta(bar_full, 0) : bar_full;
     const uint32_t acc_empty0 = TWO_SM ? map_to_cta(bar_acc_empty, 0) : bar_acc_empty;
     const uint32_t tx_mult = TWO_SM ? 2u : 1u;
+    // Global memory is read and written from here on: everything the preceding kernel wrote must be visible.
+    grid_dependency_wait();
 
     if (warp == 0 || (NPROD == 2 && warp == PROD2_WARP)) {
         // ------------------------------------------------------------------ producer (whole warp loops, one lane issues)
@@ -333,10 +338,13 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         // ------------------------------------------------------------------ epilogue: one output channel per thread
         const int quarter = warp & 3;                   // a warp may only read lanes 32*(warp%4) .. +31
         const int cgroup = (warp - 2) >> 2;             // which share of the strip's columns this warp handles
-        const int units = p.pw / SWAP_UNIT;             // 16-pixel column units: the first group takes the larger half
-        const int col_begin = cgroup == 0 ? 0 : SWAP_UNIT * ((units + 1) >> 1);
-        const int col_end = cgroup == 0 ? SWAP_UNIT * ((units + 1) >> 1) : p.pw;
+        constexpr int GROUPS = SWAP_EPI_WARPS / 4;
+        const int units = p.pw / SWAP_UNIT;             // 16-pixel column units, dealt to the groups as evenly as they go
+        const int u_base = units / GROUPS, u_rem = units % GROUPS;
+        const int col_begin = SWAP_UNIT * (cgroup * u_base + min(cgroup, u_rem));
+        const int col_end = col_begin + SWAP_UNIT * (u_base + (cgroup < u_rem ? 1 : 0));
         const int pix = swap_pixel_of_lane(lane);       // after the transpose: which pixel of each group of four this lane holds
+        const int64_t row4 = 4 * p.ldc;                 // four rows of C
         int ab = 0, cached_n_blk = -1;
         uint32_t acc_phase = 0;
         bool dead = false;
@@ -384,10 +392,12 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                     else quad_transpose<4>(out, lane);
                     if (n_quad < p.N) {                                    // N is a multiple of 4: a quad is inside or outside as a whole
                         int8_t* cp = p.C + (int64_t)(m0 + col + pix) * p.ldc + n_quad;
+                        const int rows_left = p.M - (m0 + col + pix);      // rows of C from this lane's first row to the end
 #pragma unroll
-                        for (int j = 0; j < 8; j++)
-                            if (4 * j < width && m0 + col + 4 * j + pix < p.M)
-                                *reinterpret_cast<uint32_t*>(cp + (int64_t)(4 * j) * p.ldc) = out[j];
+                        for (int j = 0; j < 8; j++) {
+                            if (4 * j < width && 4 * j < rows_left) *reinterpret_cast<uint32_t*>(cp) = out[j];
+                            cp += row4;
+                        }
                     }
                 } else if (n < p.N) {
                     int8_t* cp = p.C + (int64_t)(m0 + col) * p.ldc + n;

@@ -320,9 +320,9 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
     }
-    // Everything above touched only shared and tensor memory; from here on global memory is read and written.
+    // The next kernel of the stream may be scheduled from here on; this one goes on with set-up that touches only shared
+    // and tensor memory, and waits for its own predecessor right before the roles start (below).
     grid_launch_dependents();
-    grid_dependency_wait();
     // Set-up barrier.  The producer warp initialised the mbarriers itself and needs nothing from the others, so it
     // only signals and starts loading at once; everybody else waits for the barriers and the tensor-memory address.
     uint32_t tmem_base = 0;
@@ -356,6 +356,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const uint32_t bres0 = TWO_SM ? map_to_cta(bar_bres, 0) : bar_bres;
     const uint32_t acc_empty0 = TWO_SM ? map_to_cta(bar_acc_empty, 0) : bar_acc_empty;
     const uint32_t tx_mult = TWO_SM ? 2u : 1u;         // the even CTA's barriers count both CTAs' bytes
+    // Global memory is read and written from here on: everything the preceding kernel wrote must be visible.
+    grid_dependency_wait();
 
     if (warp == 0 || (NPROD == 2 && warp == PROD2_WARP)) {
         // ------------------------------------------------------------------ producer (whole warp loops, one lane issues)

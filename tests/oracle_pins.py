@@ -52,6 +52,127 @@ def _gemm(O, A, B, bias=None, mult=1, shift=0, relu=0, per_channel=0):
     return O.gemm_i8(As, K, 1, Bs, 1, K, N, b, mult, shift, per_channel, M, N, K, relu)
 
 
+def py_fl32(x):
+    """Round an exact rational (fractions.Fraction) to the nearest IEEE-754 binary32 value, ties to even, with Python
+    integers only (normal range; magnitudes here stay far from overflow and underflow).  Returns a Fraction."""
+    from fractions import Fraction
+    if x == 0:
+        return Fraction(0)
+    sign = -1 if x < 0 else 1
+    a = abs(Fraction(x))
+    e = a.numerator.bit_length() - a.denominator.bit_length()      # 2^e <= a < 2^(e+2): fix up below
+    if Fraction(2) ** e > a:
+        e -= 1
+    if Fraction(2) ** (e + 1) <= a:
+        e += 1
+    ulp = Fraction(2) ** (e - 23)                                  # 24 significant bits
+    q = a / ulp
+    n = q.numerator // q.denominator
+    rem = q - n
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and n % 2 == 1):
+        n += 1
+    return sign * n * ulp
+
+
+def py_rne_int(x):
+    """Nearest integer of an exact rational, ties to even."""
+    from fractions import Fraction
+    n = x.numerator // x.denominator
+    rem = x - n
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and n % 2 == 1):
+        n += 1
+    return n
+
+
+def py_requant_fscale(acc, bias, relu, scale_num, scale_log2_den):
+    """Exact-rational model of the float-scale read-out: fl32(fl32(t) * scale), nearest-even integer, clamp."""
+    from fractions import Fraction
+    t = acc + bias
+    if relu:
+        t = max(t, 0)
+    scale = Fraction(scale_num, 1 << scale_log2_den)
+    assert py_fl32(scale) == scale, "the scale must be a binary32 value"
+    y = py_fl32(py_fl32(Fraction(t)) * scale)
+    return max(-128, min(127, py_rne_int(y)))
+
+
+# ----------------------------------------------------------------------------- float-scale pins
+def pin_fscale_golden(O):
+    """Hand-derived worked values (tests/golden/fscale_worked.txt)."""
+    n = 0
+    for line in open(os.path.join(GOLDEN, "fscale_worked.txt")):
+        line = line.split("#")[0].strip()
+        if not line:
+            continue
+        acc, bias, relu, num, lg, want = (int(v) for v in line.split())
+        got, ovf = O.requant_fscale(acc, bias, relu, num / float(1 << lg))
+        assert got == want and ovf == 0, (line, got)
+        n += 1
+    assert n >= 36
+
+
+def pin_fscale_rational_model(O):
+    """Against exact rational arithmetic with explicit binary32 roundings (Python integers), over edge accumulators,
+    scales with full 24-bit mantissas and power-of-two scales; scale 1 is the saturating narrow; a power-of-two scale
+    on a small accumulator is the round-to-even of an exact quotient."""
+    accs = [0, 1, -1, 2, 3, -3, 127, 128, -128, -129, 255, 256, 1000, -1000, (1 << 23) + 1, (1 << 24) - 1, (1 << 24) + 1,
+            -(1 << 24) - 3, (1 << 25) + 6, 3 * (1 << 25) + 3, 123456789, -987654321, I32_MAX, I32_MIN, I32_MAX - 64, 16777219]
+    scales = [(1, 0), (1, 1), (3, 2), (1, 7), (5, 3), (16777215, 24), (16777215, 40), (8388609, 30), (11184811, 24), (1, 24),
+              (12345677, 44), (3, 19), (13, 30), (-3, 2), (-16777215, 31), (1, 31)]
+    rng = np.random.default_rng(11)
+    accs = accs + [int(v) for v in rng.integers(-(1 << 31), 1 << 31, size=40)] + [int(v) for v in rng.integers(-4000, 4000, size=40)]
+    for (num, lg) in scales:
+        sc = num / float(1 << lg)
+        for acc in accs:
+            for relu in (0, 1):
+                for bias in (0, -5):
+                    if not (I32_MIN <= acc + bias <= I32_MAX):
+                        continue
+                    got, _ = O.requant_fscale(acc, bias, relu, sc)
+                    assert got == py_requant_fscale(acc, bias, relu, num, lg), (acc, bias, relu, num, lg, got)
+    for t in range(-300, 300):
+        assert O.requant_fscale(t, 0, 0, 1.0)[0] == max(-128, min(127, t))
+        q, r = divmod(t, 4)                         # t / 4 = q + r/4: nearest even
+        want = q + (1 if r == 3 or (r == 2 and q % 2 == 1) else 0)
+        assert O.requant_fscale(t, 0, 0, 0.25)[0] == max(-128, min(127, want)), t
+    # monotone in t for a positive scale, antitone for a negative one; ReLU zeroes negatives; overflow flag
+    for sc in (0.37, 1.5e-3, 2.0):
+        prev = -128
+        for t in range(-2000, 2000, 7):
+            v = O.requant_fscale(t, 0, 0, sc)[0]
+            assert v >= prev
+            prev = v
+            assert O.requant_fscale(t, 0, 1, sc)[0] == (v if t >= 0 else 0)
+    assert O.requant_fscale(I32_MAX, 1, 0, 1.0)[1] == 1 and O.requant_fscale(I32_MAX, 0, 0, 1.0)[1] == 0
+
+
+def pin_fscale_gemm(O):
+    """The GEMM with the float-scale read-out: accumulators pinned by brute force elsewhere; here the read-out is applied
+    per output column with the right scale and bias (per-channel and shared), and matches the element model."""
+    rng = np.random.default_rng(12)
+    M, N, K = 5, 7, 9
+    A = rng.integers(-128, 128, size=(M, K)); B = rng.integers(-128, 128, size=(K, N))
+    acc = py_gemm_acc(A.tolist(), B.tolist())
+    bias = rng.integers(-3000, 3000, size=N).astype(np.int32)
+    nums = [3, 5, 1, 7, 11, 13, 9]; lgs = [9, 10, 8, 11, 12, 12, 10]
+    scale = np.array([n / float(1 << l) for n, l in zip(nums, lgs)], dtype=np.float32)
+    As, Bs = _row_col(A, B)
+    for relu in (0, 1):
+        C = O.gemm_i8_fscale(As, K, 1, Bs, 1, K, N, bias, scale, 1, M, N, K, relu)
+        for m in range(M):
+            for n in range(N):
+                assert C[m, n] == py_requant_fscale(acc[m][n], int(bias[n]), relu, nums[n], lgs[n]), (m, n)
+        C1 = O.gemm_i8_fscale(As, K, 1, Bs, 1, K, N, None, scale[2:3].copy(), 0, M, N, K, relu)
+        for m in range(M):
+            for n in range(N):
+                assert C1[m, n] == py_requant_fscale(acc[m][n], 0, relu, nums[2], lgs[2]), (m, n)
+    # a transposed B (swapped strides) must change the result: storage order is honoured
+    Bt = _c(B.astype(np.int8))                     # (K, N) row-major
+    C2 = O.gemm_i8_fscale(As, K, 1, Bt, N, 1, N, bias, scale, 1, M, N, K, 0)
+    C3 = O.gemm_i8_fscale(As, K, 1, Bs, 1, K, N, bias, scale, 1, M, N, K, 0)
+    assert np.array_equal(C2, C3)
+
+
 # ----------------------------------------------------------------------------- requant pins
 def pin_requant_golden(O):
     """Hand-derived worked values (tests/golden/requant_worked.txt)."""
@@ -348,6 +469,6 @@ def pin_conv_closed_forms(O):
     assert np.array_equal(part[1], full[1]) and not part[0].any() and not part[2].any()
 
 
-ALL_PINS = [pin_requant_golden, pin_requant_bigint_table, pin_requant_properties, pin_gemm_bruteforce,
+ALL_PINS = [pin_fscale_golden, pin_fscale_rational_model, pin_fscale_gemm, pin_requant_golden, pin_requant_bigint_table, pin_requant_properties, pin_gemm_bruteforce,
             pin_gemm_closed_forms, pin_gemm_symmetries, pin_gemm_epilogue_on_matrix, pin_batched,
             pin_conv_bruteforce, pin_conv_closed_forms]

@@ -88,7 +88,7 @@ def test_mpc_pins_catch_planted_mistake(label, old, new):
     with tempfile.TemporaryDirectory() as dd:
         src = os.path.join(dd, "m.c"); so = os.path.join(dd, "m.so")
         open(src, "w").write(text.replace(old, new))
-        subprocess.run(["gcc", "-O1", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", so, src], check=True)
+        subprocess.run(["gcc", "-O1", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", so, src, "-lm"], check=True)
         mutant = oracle.Oracle(so)
         caught = []
         for pin in PINS:

@@ -1,6 +1,7 @@
 """The oracle against its pins (CPU only), and the pins against deliberately broken oracles."""
 import os
 import subprocess
+import sys
 import tempfile
 
 import pytest
@@ -42,6 +43,14 @@ MUTANTS = [
     ("conv_h_w_swapped", "((int64_t)n * H + h) * W + ww) * C", "((int64_t)n * H + ww) * W + h) * C"),
     ("conv_extent_ceil", "int Q = (W + 2 * pad_w - S) / stride_w + 1;", "int Q = (W + 2 * pad_w - S + stride_w - 1) / stride_w + 1;"),
     ("conv_bound_off_by_one", "if (h < 0 || h >= H) continue;", "if (h < 0 || h >= H - 1) continue;"),
+    ("fscale_truncates", "return (int32_t)lrintf(y);", "return (int32_t)y;"),
+    ("fscale_ties_away", "return (int32_t)lrintf(y);", "return (int32_t)roundf(y);"),
+    ("fscale_double_product", "volatile float y = tf * scale;", "volatile float y = (float)((double)(int32_t)t * (double)scale);"),
+    ("fscale_relu_after_scale", "if (relu && t < 0) t = 0;\n    volatile float tf", "volatile float tf"),
+    ("fscale_bias_dropped", "int64_t t = acc + (int64_t)bias;\n    if (overflow && (t > (int64_t)INT32_MAX || t < (int64_t)INT32_MIN)) *overflow = 1;\n    if (relu && t < 0) t = 0;\n    volatile float tf",
+     "int64_t t = acc;\n    if (relu && t < 0) t = 0;\n    volatile float tf"),
+    ("fscale_clamp_hi_128", "if (y >= 127.0f) return 127;", "if (y >= 128.0f) return 128;"),
+    ("fscale_channel_index_m", "scale[per_channel ? n : 0], &ovf);", "scale[per_channel ? m : 0], &ovf);"),
     ("conv_weight_layout_kcrs", "(((int64_t)k * R + r) * S + s) * C", "(((int64_t)k * S + s) * R + r) * C"),
 ]
 
@@ -55,14 +64,16 @@ def test_pins_catch_planted_mistake(label, old, new):
         src = os.path.join(d, "oracle_mut.c")
         so = os.path.join(d, "liboracle_mut.so")
         open(src, "w").write(text.replace(old, new, 1))
-        subprocess.run(["gcc", "-O1", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", so, src], check=True)
-        mutant = oracle.Oracle(so)
-        caught = []
-        for pin in ALL_PINS:
-            try:
-                pin(mutant)
-            except AssertionError:
-                caught.append(pin.__name__)
-            except Exception:
-                caught.append(pin.__name__)
+        subprocess.run(["gcc", "-O1", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", so, src, "-lm"], check=True)
+        # The pins run in a child process: a planted indexing mistake may write outside the oracle's buffers, and a
+        # crash of the child counts as "noticed" just like a failed assertion.
+        code = ("import sys; sys.path.insert(0, %r); sys.path.insert(0, %r)\n"
+                "import oracle\nfrom oracle_pins import ALL_PINS\n"
+                "m = oracle.Oracle(%r)\n"
+                "for pin in ALL_PINS:\n"
+                "    try:\n        pin(m)\n"
+                "    except Exception:\n        sys.exit(3)\n"
+                "sys.exit(0)\n") % (os.path.dirname(HERE), HERE, so)
+        rc = subprocess.run([sys.executable, "-c", code], capture_output=True).returncode
+        caught = rc != 0
         assert caught, f"no pin noticed the planted mistake '{label}'"
