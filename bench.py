@@ -266,7 +266,7 @@ def main():
     launch(0); launch(1); launch(2)
     torch.cuda.synchronize()
     assert i8.last_device_status() == 0
-    assert i8.last_path() in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM), "the tensor path did not run"
+    assert i8.last_path() in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM, i8.PATH_CHANNEL_MAJOR, i8.PATH_CHANNEL_MAJOR_2SM), "the tensor path did not run"
     if rank == 0 and oracle_out:
         # every element of all three outputs against the oracle's
         bit_exact = all(bool(np.array_equal(dev_t[j]["C"].cpu().numpy(), oracle_out[n][:, :problems[j].N]))

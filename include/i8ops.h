@@ -267,7 +267,7 @@ int i8ops_last_path(void);
 
 /* Restrict dispatch: 0 = automatic (default), 1 = always the generic kernel, 2 = GEMMs and convolutions take the
  * two-SM tensor kernel whenever the layout allows the tensor path (also where its large tiles do not pay),
- * 3 = automatic, but stride-1 convolutions stay on the implicit-GEMM kernel instead of the slab kernel,
+ * 3 = automatic among the large-tile kernels only (no slab kernel, no channel-major kernel),
  * 4 = GEMMs and implicit-GEMM convolutions take the channel-major kernel whenever the layout allows the tensor path.
  * Returns the previous setting. */
 int i8ops_set_path(int mode);

@@ -49,7 +49,7 @@ static int g_force_bn = -1;                      // tuning override from the env
 static int g_tma_store = 1;                      // read-out of the wide tiles through TMA stores (I8OPS_TMA_STORE=0 turns it off)
 static int g_sticky = 1;                         // column-sticky tile order for short-K problems (I8OPS_STICKY=0 turns it off)
 static int g_tmap_cache = 1;                     // per-thread cache of encoded tensor maps (I8OPS_TMAP_CACHE=0 encodes every time)
-static int g_swap = 0;                           // channel-major kernel: 0 never, 1 by rule, 2 wherever legal (I8OPS_SWAP)
+static int g_swap = 1;                           // channel-major kernel: 0 never, 1 by rule, 2 wherever legal (I8OPS_SWAP)
 static int g_swap_stages = 0;                    // ring slots of the channel-major kernel: 0 = as many as fit (I8OPS_SWAP_STAGES)
 static int g_swap_pw = 0;                        // strip width override for tuning (I8OPS_SWAP_PW)
 static int g_slab = 1;                           // slab-resident stride-1 convolution kernel (I8OPS_SLAB=0 turns it off)
@@ -507,7 +507,7 @@ static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap
 static int run_gemm_swap(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                          const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N, int K,
                          int relu, cudaStream_t st);
-static bool swap_wanted(int M, int N, int num_kb, int sm_count);
+static bool swap_wanted(bool conv, int M, int N, int K, int num_kb, int num_iters, int num_kblocks, int cb, int sm_count);
 
 static KLoop gemm_kloop(int K) {
     KLoop kl{};
@@ -524,7 +524,7 @@ static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_
     KLoop kl = gemm_kloop(K);
     kl.a_mn = a_mn; kl.b_mn = b_mn;
     t_used_swap = false;
-    if (!raw.D && !a_mn && !b_mn && swap_wanted(M, N, kl.num_kblocks, ctx->sm_count)) {
+    if (!raw.D && !a_mn && !b_mn && swap_wanted(false, M, N, K, kl.num_kblocks, kl.num_iters, kl.num_kblocks, BK, ctx->sm_count)) {
         int rc = run_gemm_swap(ctx, A, lda, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
         if (rc != I8_ERR_UNSUPPORTED) { t_used_swap = rc == I8_OK; return rc; }
     }
@@ -635,12 +635,25 @@ static int run_swap(DeviceCtx* ctx, bool conv, const SwapPlan& pl, const CUtenso
 }
 
 // Whether a problem goes to the channel-major kernel.  Forced (path mode 4, I8OPS_SWAP=2): whenever it is legal.  By
-// rule: problems too small for the 256 x 256 pair kernel to pay, with at least 128 output channels.
-static bool swap_wanted(int M, int N, int num_kb, int sm_count) {
+// rule: its read-out costs more per output than the large-tile kernel's (a transpose in registers), so it is taken only
+// where its freely chosen strip width buys occupancy: the large-tile plan would leave at least a fifth more of the chip
+// idle than the channel-major plan (the 3x3 layers with 12544 pixels and 256 filters: 98 tiles on 148 SMs against 72
+// strips on 74 CTA pairs; measured 8.6 -> 8.0 us and 11.4 -> 9.9 us), on problems with enough K per tile for that to
+// matter and too small for the 256 x 256 pair kernel.
+static bool swap_wanted(bool conv, int M, int N, int K, int num_kb, int num_iters, int num_kblocks, int cb, int sm_count) {
     if (g_path_mode == 4 || g_swap == 2) return true;
     if (!g_swap || g_path_mode != 0 || g_force_bn >= 0) return false;
-    if (N < 128) return false;
-    return !(g_tc2 && pair_pays(M, N, 256, num_kb, sm_count));
+    if (N < 256 || num_iters < 8) return false;
+    if (!conv && recorded_plan(M, N, K)) return false;      // a schedule recorded for this shape's class takes precedence
+    const TcPlan old_plan = plan_tc(conv, M, N, K, num_kb, num_iters, num_kblocks, cb, sm_count);
+    if (old_plan.two_sm || 2 * old_plan.num_tiles < sm_count) return false;   // tiny problems: launch latency, not occupancy, bounds them
+    const SwapPlan sp = plan_swap(M, N, num_iters, true, sm_count);
+    if (!sp.pw) return false;
+    const int waves_old = (old_plan.num_tiles + sm_count - 1) / sm_count;
+    const double eff_old = (double)old_plan.num_tiles / ((double)waves_old * sm_count);
+    const int pairs = sm_count / 2, waves_new = (sp.num_tiles + pairs - 1) / pairs;
+    const double eff_new = (double)sp.num_tiles / ((double)waves_new * pairs);
+    return eff_new - eff_old >= 0.2;
 }
 
 static int run_gemm_swap(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
@@ -674,7 +687,7 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     kl.stride_h = stride_h; kl.stride_w = stride_w; kl.pad_h = pad_h; kl.pad_w = pad_w;
     const int K = R * S * C;
     t_used_swap = false;
-    if (swap_wanted(M, Kf, (K + BK - 1) / BK, ctx->sm_count)) {
+    if (swap_wanted(true, M, Kf, K, (K + BK - 1) / BK, kl.num_iters, kl.num_kblocks, cb, ctx->sm_count)) {
         // filters on the tensor-memory lanes, a strip of output pixels on the columns
         const SwapPlan sp = plan_swap(M, Kf, kl.num_iters, Kf > 128, ctx->sm_count);
         if (sp.pw && sp.stages >= 2) {

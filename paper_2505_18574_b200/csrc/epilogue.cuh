@@ -116,41 +116,6 @@ __device__ __forceinline__ uint32_t relu_s8x4(uint32_t x) {
     return x & ~neg;
 }
 
-// ---------------------------------------------------------------------------------------------------------
-// Double-precision form.  The 64-bit integer multiply-add above is the slowest instruction of the read-out (measured on
-// B200: about 12 results per clock per SM), while the FP64 pipe retires 64 fused multiply-adds per clock per SM.  For
-// |mult| < 2^20 every quantity of the definition is an integer below 2^52, so doubles hold it exactly:
-//   T  = the double whose bit pattern is (0x43300000, acc ^ 0x80000000) = 2^52 + 2^31 + acc            (one logic op)
-//   td = T - kb,  kb = 2^52 + 2^31 - bias                      = acc + bias, exact (one FP64 add)
-//   z  = fma_round_down(td, ms, 1.5 * 2^51 + 0.5),  ms = mult * 2^-shift (exact: a power-of-two scaling)
-// The exact value of the fused product-sum is t*mult/2^shift + 0.5 + 1.5*2^51 with |t*mult| < 2^51; doubles in
-// [2^51, 2^52) are the multiples of 0.5, so rounding down yields z = 1.5*2^51 + h with h = the largest multiple of 0.5
-// not above u = t*mult/2^shift + 0.5, and floor(h) = floor(u) = floor((t*mult + 2^(shift-1)) / 2^shift), the wanted
-// result.  The mantissa of z is 2^51 + 2h, whose low 32 bits are 2h as a two's-complement number as long as
-// |h| < 2^30: guaranteed by -2^(shift-1) < mult < 2^(shift-1) (a scale below one half) since |t| <= 2^31.  So
-// result = (low word of z) >> 1 (arithmetic), and the saturating pack finishes the clamp.  Two FP64 operations and two
-// integer operations per output.  ReLU is applied to the packed bytes afterwards, which is exact for mult >= 0 (the
-// scaled value of a negative sum is <= 0 either way); channels with ReLU and a negative multiplier use another form.
-struct F64Const {
-    double ms;      // mult * 2^-shift
-    double kb;      // 2^52 + 2^31 - bias
-};
-__device__ __forceinline__ bool make_f64_const(int32_t bias, int32_t mult, int32_t shift, int relu, F64Const& c) {
-    c.ms = 0.0;
-    c.kb = 4503601774854144.0 - (double)bias;                 // 2^52 + 2^31 - bias, exact
-    if (shift < 1) return false;
-    const int32_t half = 1 << (shift - 1);
-    if (mult <= -half || mult >= half || mult <= -(1 << 20) || mult >= (1 << 20)) return false;
-    if (relu && mult < 0) return false;
-    c.ms = __hiloint2double((1023 - shift) << 20, 0) * (double)mult;   // 2^-shift * mult
-    return true;
-}
-__device__ __forceinline__ int32_t requant_f64(int32_t acc, const F64Const& c) {
-    const double t = __hiloint2double(0x43300000, acc ^ (int32_t)0x80000000) - c.kb;
-    const double z = __fma_rd(t, c.ms, 3377699720527872.5);   // 1.5 * 2^51 + 0.5
-    return __double2loint(z) >> 1;
-}
-
 // Saturate four 32-bit values to int8 and pack them, v0 in the lowest byte.
 // cvt.pack.sat.s8.s32.b32 d, a, b, c  gives  d = (c << 16) | (sat8(a) << 8) | sat8(b).
 __device__ __forceinline__ uint32_t pack_sat4(int32_t v0, int32_t v1, int32_t v2, int32_t v3) {

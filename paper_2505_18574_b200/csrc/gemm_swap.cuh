@@ -58,18 +58,18 @@ struct SwapParams {
 // Per-thread epilogue constants of one output channel.
 struct SwapChan {
     int32_t bias, m2;
-    F64Const f64;
+    long long c64;
     ChanConst cc;
-    int form;                   // 0 double-precision form, 1 shift-32 form (ReLU ahead of the scale), 2 window form
+    int form;                   // 0 folded shift-32 form, 1 shift-32 form with ReLU ahead of the scale, 2 window form
 };
 
 __device__ __forceinline__ SwapChan make_swap_chan(int32_t bias, int32_t mult, int32_t shift, int relu) {
     SwapChan c;
     c.bias = bias;
     const bool ok32 = make_shift32_mult(mult, shift, c.m2);
-    const bool ok64 = make_f64_const(bias, mult, shift, relu, c.f64);
+    c.c64 = make_fold_addend(bias, c.m2);
     c.cc = make_chan_const(mult, shift, relu);
-    c.form = ok64 ? 0 : (ok32 ? 1 : 2);
+    c.form = ok32 ? ((!relu || c.m2 >= 0) ? 0 : 1) : 2;
     return c;
 }
 
@@ -79,22 +79,15 @@ __device__ __forceinline__ void swap_requant(const int32_t (&v)[32], const SwapC
     if (ch.form == 0) {
 #pragma unroll
         for (int j = 0; j < COUNT / 4; j++) {
-            const uint32_t pk = pack_sat4(requant_f64(v[4 * j + 0], ch.f64), requant_f64(v[4 * j + 1], ch.f64),
-                                          requant_f64(v[4 * j + 2], ch.f64), requant_f64(v[4 * j + 3], ch.f64));
+            const uint32_t pk = pack_sat4(requant_fold(v[4 * j + 0], ch.m2, ch.c64), requant_fold(v[4 * j + 1], ch.m2, ch.c64),
+                                          requant_fold(v[4 * j + 2], ch.m2, ch.c64), requant_fold(v[4 * j + 3], ch.m2, ch.c64));
             out[j] = relu ? relu_s8x4(pk) : pk;
         }
     } else if (ch.form == 1) {
-        if (relu) {
 #pragma unroll
-            for (int j = 0; j < COUNT / 4; j++)
-                out[j] = pack_sat4(requant_shift32<true>(v[4 * j + 0], ch.bias, ch.m2), requant_shift32<true>(v[4 * j + 1], ch.bias, ch.m2),
-                                   requant_shift32<true>(v[4 * j + 2], ch.bias, ch.m2), requant_shift32<true>(v[4 * j + 3], ch.bias, ch.m2));
-        } else {
-#pragma unroll
-            for (int j = 0; j < COUNT / 4; j++)
-                out[j] = pack_sat4(requant_shift32<false>(v[4 * j + 0], ch.bias, ch.m2), requant_shift32<false>(v[4 * j + 1], ch.bias, ch.m2),
-                                   requant_shift32<false>(v[4 * j + 2], ch.bias, ch.m2), requant_shift32<false>(v[4 * j + 3], ch.bias, ch.m2));
-        }
+        for (int j = 0; j < COUNT / 4; j++)
+            out[j] = pack_sat4(requant_shift32<true>(v[4 * j + 0], ch.bias, ch.m2), requant_shift32<true>(v[4 * j + 1], ch.bias, ch.m2),
+                               requant_shift32<true>(v[4 * j + 2], ch.bias, ch.m2), requant_shift32<true>(v[4 * j + 3], ch.bias, ch.m2));
     } else {
 #pragma unroll
         for (int j = 0; j < COUNT / 4; j++)

@@ -24,11 +24,11 @@ def _conv_both(p, expect_tensor=None):
     path = i8.last_path()
     H.assert_same(got, want, f"{p.name} auto path={path}")
     if expect_tensor is not None:
-        assert (path in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM, i8.PATH_CONV_SLAB)) == expect_tensor, f"{p.name}: path {path}"
-    if path == i8.PATH_CONV_SLAB:
-        i8.set_path(3)                                   # the same layer without the slab kernel
+        assert (path in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM, i8.PATH_CONV_SLAB, i8.PATH_CHANNEL_MAJOR, i8.PATH_CHANNEL_MAJOR_2SM)) == expect_tensor, f"{p.name}: path {path}"
+    if path in (i8.PATH_CONV_SLAB, i8.PATH_CHANNEL_MAJOR, i8.PATH_CHANNEL_MAJOR_2SM):
+        i8.set_path(3)                                   # the same layer on the large-tile implicit-GEMM kernel
         got = H.conv_gpu(p)
-        assert i8.last_path() != i8.PATH_CONV_SLAB, f"{p.name}: path {i8.last_path()}"
+        assert i8.last_path() in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM, i8.PATH_GENERIC), f"{p.name}: path {i8.last_path()}"
         H.assert_same(got, want, f"{p.name} implicit GEMM (or generic, for small activations)")
     i8.set_path(1)
     got = H.conv_gpu(p)

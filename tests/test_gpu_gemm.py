@@ -16,7 +16,7 @@ def _auto_path():
     i8.set_path(0)
 
 
-TENSOR_PATHS = (2, 4)      # one-SM and two-SM tensor kernels
+TENSOR_PATHS = (2, 4, 6, 7)      # large-tile kernel on one CTA / CTA pairs, channel-major kernel on one CTA / CTA pairs
 
 
 def _both_paths(p, expect_tensor=True, two_sm=False):

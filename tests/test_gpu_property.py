@@ -56,9 +56,9 @@ def test_random_convs(N, H_, W, C32, K, R, stride, pad, seed, relu):
     i8.set_path(0)
     got = H.conv_gpu(p)
     path = i8.last_path()
-    assert path in (i8.PATH_TENSOR, i8.PATH_CONV_SLAB)
+    assert path in (i8.PATH_TENSOR, i8.PATH_CONV_SLAB, i8.PATH_CHANNEL_MAJOR, i8.PATH_CHANNEL_MAJOR_2SM)
     H.assert_same(got, want, f"{p.name} seed {seed} path {path}")
-    if path == i8.PATH_CONV_SLAB:                       # stride-1 layers with few filters: also the implicit-GEMM kernel
+    if path != i8.PATH_TENSOR:                          # also the large-tile implicit-GEMM kernel
         i8.set_path(3)
         got = H.conv_gpu(p)
         assert i8.last_path() == i8.PATH_TENSOR
