@@ -332,6 +332,26 @@ def main():
     d2h = sum(p.M * p.N for p in problems)
     e2e_exact = all(np.array_equal(host[j]["C"].numpy(), dev_t[j]["C"].cpu().numpy()) for j in range(3))
 
+    # Strong scaling beside the per-rank replicas (several GPUs only): ONE 16384 x 4096 x 8192 problem, its rows split
+    # across the ranks (no exchange step; every rank holds B), timed on the device as the max over ranks.
+    strong = None
+    if world > 1:
+        p2, d2 = problems[2], dev_t[2]
+        call = lambda: sharding.sharded_gemm_i8(d2["A"], d2["B"].t(), d2["bias"], d2["mult"], d2["shift"], p2.per_channel, p2.relu,
+                                                world=world, rank=rank, out=d2["C"][:sharding.row_shard(p2.M, world, rank)[1]])
+        for _ in range(3):
+            call()
+        barrier()
+        s0 = torch.cuda.Event(enable_timing=True); s1 = torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for _ in range(20):
+            call()
+        s1.record()
+        barrier()
+        ms = sharding.max_over_ranks(s0.elapsed_time(s1) / 20, dev)
+        strong = {"problem": p2.name, "rows_per_rank": sharding.row_shard(p2.M, world, 0)[1], "ms": ms, "tops": gemm_ops(p2) / (ms * 1e-3) / 1e12,
+                  "scaling": "strong"}
+
     details, probe = None, None
     if rank == 0 and world == 1:
         from paper_2505_18574_b200 import bench_details
@@ -397,6 +417,8 @@ def main():
                        "samples": clocks["samples"], "window": clocks["window"]},
             "bit_exact_vs_oracle": bit_exact,
         }
+        if strong is not None:
+            line["strong_scaling_row_sharded"] = strong
         if cpu_baseline is not None:
             line["cpu_baseline"] = cpu_baseline
         if details is not None:

@@ -104,6 +104,22 @@ int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs,
                 int M, int N, int K, void* stream);
 
 /*
+ * gemm_i8 with the read-out scale given as a single-precision float, as the paper's Gemmini listings pass it (the scale
+ * argument of the ISA description's store configuration, 1.0f in the printed GEMM):
+ *     t = acc + bias[n];  t = max(t, 0) if relu;  out = min(127, max(-128, rne(fl32(fl32(t) * scale[n]))))
+ * fl32 = rounding to IEEE-754 binary32 (nearest, ties to even), applied to the conversion of t and to the product;
+ * rne = nearest integer, ties to even (the paper states no rounding rule; this is the reading taken).  A NaN product
+ * yields 0.  scale: device, float[1] (per_channel == 0) or float[N].  Other arguments, layouts and errors as gemm_i8
+ * (I8_ERR_NULL also for a NULL scale).  K-contiguous aligned operands run on the channel-major tensor kernel, anything
+ * else on the generic kernel.
+ */
+int gemm_i8_fscale(const int8_t* A, int64_t a_rs, int64_t a_cs,
+                   const int8_t* B, int64_t b_rs, int64_t b_cs,
+                   int8_t* C, int64_t ldc,
+                   const int32_t* bias, const float* scale, int per_channel,
+                   int M, int N, int K, int relu, void* stream);
+
+/*
  * `batch` independent products (the paper's fine-grained linear algebra: many small, low-reuse
  * products, Evaluation "Fine-Grained Linear Algebra"; also its column-dominant GEMM shapes).
  * Problem b uses A + b*a_bs, B + b*b_bs, C + b*c_bs and bias + b*bias_bs (bias_bs == 0: one bias

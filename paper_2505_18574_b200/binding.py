@@ -25,6 +25,7 @@ _int = ctypes.c_int
 SIGNATURES = {
     "gemm_i8": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
     "gemm_i8_raw": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _int, _int, _int, _int, _vp]),
+    "gemm_i8_fscale": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
     "batched_gemm_i8": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _int,
                                _int, _int, _int, _int, _int, _vp]),
     "conv2d_i8": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int] + [_int] * 12 + [_vp]),
@@ -114,6 +115,16 @@ def gemm_i8_raw(A, B, D, accumulate: bool = False, stream=None) -> None:
     st = lib().gemm_i8_raw(_ptr(A), A.stride(0), A.stride(1), _ptr(B), B.stride(0), B.stride(1), _ptr(D), D.stride(0),
                            int(bool(accumulate)), M, N, K, _stream_ptr(stream))
     _check(st, "gemm_i8_raw")
+
+
+def gemm_i8_fscale(A, B, C, bias, scale, per_channel: int, relu: int, stream=None) -> None:
+    """C = float-scale read-out of A . B (see ``gemm_i8_fscale`` in i8ops.h); scale: float32 CUDA tensor, [1] or [N]."""
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2 and tuple(C.shape) == (M, N) and (C.stride(1) == 1 or N <= 1)
+    st = lib().gemm_i8_fscale(_ptr(A), A.stride(0), A.stride(1), _ptr(B), B.stride(0), B.stride(1), _ptr(C), C.stride(0),
+                              _ptr(bias), _ptr(scale), int(per_channel), M, N, K, int(relu), _stream_ptr(stream))
+    _check(st, "gemm_i8_fscale")
 
 
 def _batched_gemm_i8_args(A, B, C, bias, mult, shift, per_channel, relu, stream=None):

@@ -506,7 +506,7 @@ static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap
 
 static int run_gemm_swap(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                          const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N, int K,
-                         int relu, cudaStream_t st);
+                         int relu, cudaStream_t st, const float* fscale = nullptr);
 static bool swap_wanted(bool conv, int M, int N, int K, int num_kb, int num_iters, int num_kblocks, int cb, int sm_count);
 
 static KLoop gemm_kloop(int K) {
@@ -607,7 +607,7 @@ static int launch_swap(DeviceCtx* ctx, int slot, const SwapPlan& pl, const CUten
 // plan's b_rows.  C row-major [M][ldc].
 static int run_swap(DeviceCtx* ctx, bool conv, const SwapPlan& pl, const CUtensorMap& tmX, const KLoop& kl, const int8_t* W, int64_t ldw,
                     int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
-                    int M, int N, int K, int relu, cudaStream_t st) {
+                    int M, int N, int K, int relu, cudaStream_t st, const float* fscale = nullptr) {
     CUtensorMap tmW;
     {
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
@@ -618,6 +618,7 @@ static int run_swap(DeviceCtx* ctx, bool conv, const SwapPlan& pl, const CUtenso
     }
     SwapParams p;
     p.C = C; p.ldc = ldc; p.bias = bias; p.mult = mult; p.shift = shift; p.per_channel = per_channel; p.relu = relu;
+    p.fscale = fscale;
     p.M = M; p.N = N; p.K = K;
     p.pw = pl.pw; p.b_rows = pl.b_rows;
     p.c_word_ok = ((reinterpret_cast<uintptr_t>(C) & 3u) == 0 && ldc % 4 == 0 && N % 4 == 0) ? 1 : 0;
@@ -658,7 +659,7 @@ static bool swap_wanted(bool conv, int M, int N, int K, int num_kb, int num_iter
 
 static int run_gemm_swap(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, int8_t* C, int64_t ldc,
                          const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N, int K,
-                         int relu, cudaStream_t st) {
+                         int relu, cudaStream_t st, const float* fscale) {
     const KLoop kl = gemm_kloop(K);
     const SwapPlan pl = plan_swap(M, N, kl.num_iters, N > 128, ctx->sm_count);
     if (!pl.pw || pl.stages < 2) return I8_ERR_UNSUPPORTED;
@@ -668,7 +669,7 @@ static int run_gemm_swap(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int
     const uint32_t box[2] = {BK, (uint32_t)pl.b_rows};
     int rc = make_tmap(&tmX, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
-    return run_swap(ctx, false, pl, tmX, kl, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
+    return run_swap(ctx, false, pl, tmX, kl, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, fscale);
 }
 
 // Implicit-GEMM convolution: A tiles come from an im2col-mode tensor map over the NHWC activations.
@@ -905,6 +906,34 @@ int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, in
     }
     GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, nullptr, 0, 0, nullptr, 0, nullptr, nullptr, 0, 0, 1, M, N, K,
                         D, ldd, 1, accumulate ? 1 : 0};
+    rc = run_gemm_generic(g, st);
+    if (rc == I8_OK) t_last_path = I8_PATH_GENERIC;
+    return rc;
+}
+
+int gemm_i8_fscale(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_t b_rs, int64_t b_cs, int8_t* C, int64_t ldc,
+                   const int32_t* bias, const float* scale, int per_channel, int M, int N, int K, int relu, void* stream) {
+    t_last_path = I8_PATH_NONE;
+    if (M < 0 || N < 0 || K < 0) return I8_ERR_SHAPE;
+    if (K > 65536) return I8_ERR_RANGE;
+    if (M == 0 || N == 0) return I8_OK;
+    if (!C || !scale || (K > 0 && (!A || !B))) return I8_ERR_NULL;
+    if (!strides_ok(a_rs, a_cs, M, K) || !strides_ok(b_rs, b_cs, K, N) || ldc < N) return I8_ERR_STRIDE;
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    // tensor path: the channel-major kernel (every thread owns one output channel, so the scale is one register)
+    const bool tc_legal = K >= 1 && a_cs == 1 && b_rs == 1 && aligned16(A) && aligned16(B) && a_rs % 16 == 0 && b_cs % 16 == 0 &&
+                          a_rs >= K && b_cs >= K;
+    if (tc_legal && g_path_mode != 1) {
+        t_used_two_sm = false; t_tmap_failed = false;
+        rc = run_gemm_swap(ctx, A, a_rs, B, b_cs, C, ldc, bias, nullptr, nullptr, per_channel, M, N, K, relu, st, scale);
+        if (rc == I8_OK) { t_used_swap = true; t_last_path = tensor_path_used(); return rc; }
+        if (rc != I8_ERR_UNSUPPORTED && !(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
+    }
+    GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, C, ldc, 0, bias, 0, nullptr, nullptr, per_channel, relu, 1, M, N, K,
+                        nullptr, 0, 0, 0, scale};
     rc = run_gemm_generic(g, st);
     if (rc == I8_OK) t_last_path = I8_PATH_GENERIC;
     return rc;

@@ -116,6 +116,15 @@ __device__ __forceinline__ uint32_t relu_s8x4(uint32_t x) {
     return x & ~neg;
 }
 
+// Float-scale read-out (the scale as the single-precision float that the paper's Gemmini listings pass to the store
+// configuration): binary32 arithmetic, out = clamp(rne(fl32(fl32(t) * scale))).  The conversion saturates to int32 and
+// the caller's saturating pack finishes the clamp; a NaN product converts to 0.
+__device__ __forceinline__ int32_t requant_fscale(int32_t acc, int32_t bias, int relu, float scale) {
+    int32_t t = acc + bias;
+    if (relu) t = max(t, 0);
+    return __float2int_rn(__fmul_rn(__int2float_rn(t), scale));
+}
+
 // Saturate four 32-bit values to int8 and pack them, v0 in the lowest byte.
 // cvt.pack.sat.s8.s32.b32 d, a, b, c  gives  d = (c << 16) | (sat8(a) << 8) | sat8(b).
 __device__ __forceinline__ uint32_t pack_sat4(int32_t v0, int32_t v1, int32_t v2, int32_t v3) {

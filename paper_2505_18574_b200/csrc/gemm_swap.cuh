@@ -39,6 +39,7 @@ struct SwapParams {
     const int32_t* bias;
     const int32_t* mult;
     const int32_t* shift;
+    const float* fscale;        // non-NULL: float-scale read-out (one entry or N), mult / shift unused
     int per_channel, relu;
     int M, N, K;
     int pw;                     // strip width: rows of C per tile, a multiple of 16, at most 256
@@ -60,7 +61,8 @@ struct SwapChan {
     int32_t bias, m2;
     long long c64;
     ChanConst cc;
-    int form;                   // 0 folded shift-32 form, 1 shift-32 form with ReLU ahead of the scale, 2 window form
+    float fscale;
+    int form;                   // 0 folded shift-32 form, 1 shift-32 form with ReLU ahead of the scale, 2 window form, 3 float scale
 };
 
 __device__ __forceinline__ SwapChan make_swap_chan(int32_t bias, int32_t mult, int32_t shift, int relu) {
@@ -70,6 +72,7 @@ __device__ __forceinline__ SwapChan make_swap_chan(int32_t bias, int32_t mult, i
     c.c64 = make_fold_addend(bias, c.m2);
     c.cc = make_chan_const(mult, shift, relu);
     c.form = ok32 ? ((!relu || c.m2 >= 0) ? 0 : 1) : 2;
+    c.fscale = 0.f;
     return c;
 }
 
@@ -88,6 +91,11 @@ __device__ __forceinline__ void swap_requant(const int32_t (&v)[32], const SwapC
         for (int j = 0; j < COUNT / 4; j++)
             out[j] = pack_sat4(requant_shift32<true>(v[4 * j + 0], ch.bias, ch.m2), requant_shift32<true>(v[4 * j + 1], ch.bias, ch.m2),
                                requant_shift32<true>(v[4 * j + 2], ch.bias, ch.m2), requant_shift32<true>(v[4 * j + 3], ch.bias, ch.m2));
+    } else if (ch.form == 3) {
+#pragma unroll
+        for (int j = 0; j < COUNT / 4; j++)
+            out[j] = pack_sat4(requant_fscale(v[4 * j + 0], ch.bias, relu, ch.fscale), requant_fscale(v[4 * j + 1], ch.bias, relu, ch.fscale),
+                               requant_fscale(v[4 * j + 2], ch.bias, relu, ch.fscale), requant_fscale(v[4 * j + 3], ch.bias, relu, ch.fscale));
     } else {
 #pragma unroll
         for (int j = 0; j < COUNT / 4; j++)
@@ -349,12 +357,14 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                 // this thread's channel changed: three loads, before the wait so that they overlap the main loop
                 n = n_blk * TILE_CH + (int)rank * BM + quarter * 32 + lane;
                 int32_t bias = 0, mult = 0, shift = 0;
+                float fs = 0.f;
                 if (n < p.N) {
                     bias = p.bias ? p.bias[n] : 0;
-                    mult = p.mult[p.per_channel ? n : 0];
-                    shift = p.shift[p.per_channel ? n : 0];
+                    if (p.fscale) fs = p.fscale[p.per_channel ? n : 0];
+                    else { mult = p.mult[p.per_channel ? n : 0]; shift = p.shift[p.per_channel ? n : 0]; }
                 }
                 ch = make_swap_chan(bias, mult, shift, p.relu);
+                if (p.fscale) { ch.form = 3; ch.fscale = fs; }
                 cached_n_blk = n_blk;
             }
             if (!dead) dead = !__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * ab, acc_phase, env, DEV_TIMEOUT_EPILOGUE));

@@ -16,6 +16,7 @@ struct GenericGemmParams {
     int per_channel, relu;
     int batch, M, N, K;
     int32_t* D; int64_t ldd; int raw, accumulate;   // raw read-out of the accumulators (see gemm_i8_raw)
+    const float* fscale;                            // non-NULL: float-scale read-out (see gemm_i8_fscale)
 };
 
 __global__ void __launch_bounds__(256) gemm_i8_generic_kernel(const GenericGemmParams p) {
@@ -36,6 +37,11 @@ __global__ void __launch_bounds__(256) gemm_i8_generic_kernel(const GenericGemmP
         }
         const int32_t bias = p.bias ? p.bias[b * p.bias_bs + n] : 0;
         const int ci = p.per_channel ? n : 0;
+        if (p.fscale) {
+            const int32_t r = requant_fscale(acc, bias, p.relu, p.fscale[ci]);
+            p.C[b * p.c_bs + (int64_t)m * p.ldc + n] = (int8_t)min(127, max(-128, r));
+            continue;
+        }
         p.C[b * p.c_bs + (int64_t)m * p.ldc + n] = (int8_t)requant_wide(acc, bias, p.relu, p.mult[ci], p.shift[ci]);
     }
 }

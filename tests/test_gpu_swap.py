@@ -122,3 +122,39 @@ def test_config3_conv_mix_channel_major(j):
     assert i8.last_path() == i8.PATH_CHANNEL_MAJOR_2SM
     H.assert_same(got, want, p.name)
     H.not_degenerate(want)
+
+
+@pytest.mark.parametrize("M,N,K,per_channel,relu", [(300, 200, 112, 1, 0), (1000, 520, 272, 1, 1), (64, 40, 48, 0, 1), (2048, 256, 1024, 1, 0),
+                                                    (129, 257, 33, 0, 0)])
+def test_float_scale_readout(M, N, K, per_channel, relu):
+    """gemm_i8_fscale (the scale as a binary32 float, round to nearest even) against its oracle, on the tensor path and on
+    the generic kernel; scales with full mantissas so that both binary32 roundings matter."""
+    import torch
+    import oracle
+    import paper_2505_18574_b200 as i8
+    pad = (-K) % 16
+    p = inputs.make_gemm(M, N, K, 6400 + M + N, per_channel=per_channel, relu=relu, lda_pad=pad, ldb_pad=pad)
+    rng = np.random.default_rng(M + N)
+    nq = N if per_channel else 1
+    scale = (rng.uniform(0.5, 1.0, size=nq) * 2.0 ** rng.integers(-14, -8, size=nq)).astype(np.float32)
+    scale[::5] *= -1.0
+    want = oracle.gemm_i8_fscale(p.A, p.a_rs, 1, p.B, 1, p.b_cs, N, p.bias, scale, per_channel, M, N, K, relu)
+    A = torch.from_numpy(p.A).cuda()[:, :K]; B = torch.from_numpy(p.B).cuda()[:, :K]
+    bias = torch.from_numpy(p.bias).cuda(); sc = torch.from_numpy(scale).cuda()
+    for mode in (0, 1):
+        i8.set_path(mode)
+        C = torch.full((M, N), 0x5A, dtype=torch.int8, device="cuda")
+        i8.gemm_i8_fscale(A, B.t(), C, bias, sc, per_channel, relu)
+        assert i8.last_device_status() == 0
+        assert i8.last_path() == (i8.PATH_GENERIC if mode == 1 else (i8.PATH_CHANNEL_MAJOR_2SM if N > 128 else i8.PATH_CHANNEL_MAJOR))
+        H.assert_same(C.cpu().numpy(), want, f"float scale mode {mode}")
+    H.not_degenerate(want)
+    # large accumulators: |t| above 2^24 is rounded by the conversion itself
+    p.A[:] = 127; p.B[:] = 127
+    A = torch.from_numpy(p.A).cuda()[:, :K]; B = torch.from_numpy(p.B).cuda()[:, :K]
+    big = np.full(nq, 1.0 / (127 * 127 * K) * 100.3, dtype=np.float32)
+    want = oracle.gemm_i8_fscale(p.A, p.a_rs, 1, p.B, 1, p.b_cs, N, p.bias, big, per_channel, M, N, K, relu)
+    i8.set_path(0)
+    C = torch.empty((M, N), dtype=torch.int8, device="cuda")
+    i8.gemm_i8_fscale(A, B.t(), C, bias, torch.from_numpy(big).cuda(), per_channel, relu)
+    H.assert_same(C.cpu().numpy(), want, "float scale, constant operands")
