@@ -966,6 +966,26 @@ int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs, c
             if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
     }
+    // Larger problems: one launch of the large-tile (or channel-major) kernel per problem, when each problem is big enough
+    // to be worth a launch of its own (128^3 multiply-accumulates, or a short batch) and every slice keeps the alignment
+    // the tensor path needs.
+    if (g_path_mode != 1 && K >= 1 && ((int64_t)M * N * K >= (1ll << 21) || batch <= 8) && batch <= 65536) {
+        const bool a_k = a_cs == 1 && a_rs % 16 == 0 && a_rs >= K, a_m = !a_k && a_rs == 1 && a_cs % 16 == 0 && a_cs >= M;
+        const bool b_k = b_rs == 1 && b_cs % 16 == 0 && b_cs >= K, b_n = !b_k && b_cs == 1 && b_rs % 16 == 0 && b_rs >= N;
+        if (aligned16(A) && aligned16(B) && a_bs % 16 == 0 && b_bs % 16 == 0 && (a_k || a_m) && (b_k || b_n)) {
+            int last = I8_PATH_NONE;
+            for (int b = 0; b < batch; b++) {
+                t_used_two_sm = false; t_tmap_failed = false;
+                rc = run_gemm_tc(ctx, A + (int64_t)b * a_bs, a_k ? a_rs : a_cs, B + (int64_t)b * b_bs, b_k ? b_cs : b_rs, C + (int64_t)b * c_bs, ldc,
+                                 bias ? bias + (int64_t)b * bias_bs : nullptr, mult, shift, per_channel, M, N, K, relu, st, RawOut(),
+                                 a_m ? 1 : 0, b_n ? 1 : 0);
+                if (rc == I8_ERR_CUDA && t_tmap_failed && b == 0) break;        // no tensor map for this geometry: generic kernel below
+                if (rc) return rc;
+                last = tensor_path_used();
+            }
+            if (rc == I8_OK) { t_last_path = last; return rc; }
+        }
+    }
     GenericGemmParams g{A, a_rs, a_cs, a_bs, B, b_rs, b_cs, b_bs, C, ldc, c_bs, bias, bias_bs, mult, shift, per_channel, relu,
                         batch, M, N, K, nullptr, 0, 0, 0};
     rc = run_gemm_generic(g, st);

@@ -197,6 +197,23 @@ def test_batched_shapes(batch, M, N, K, ppb):
     for mode in (0, 1):
         i8.set_path(mode)
         H.assert_same(H.batched_gpu(p), want, f"{p.name} mode {mode}")
+        if mode == 0 and M % 16 == 0 and N % 16 == 0 and K % 16 == 0:
+            assert i8.last_path() != i8.PATH_GENERIC, "aligned problems run on a tensor path, whatever their size"
+
+
+@pytest.mark.parametrize("batch,M,N,K", [(3, 128, 128, 128), (5, 256, 192, 320), (2, 130, 144, 80), (40, 128, 128, 128), (4, 1024, 512, 256)])
+def test_batched_problems_larger_than_the_paired_tile(batch, M, N, K):
+    """Problems above 64 in any dimension: one launch of the large-tile kernel per problem (row-major B through the MN-major
+    descriptor), per-problem bias."""
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_batched(batch, M, N, K, 700 + batch + M + N)
+    p.shift[:] = 24
+    want = H.batched_oracle(p)
+    i8.set_path(0)
+    got = H.batched_gpu(p)
+    assert i8.last_path() in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM, i8.PATH_CHANNEL_MAJOR, i8.PATH_CHANNEL_MAJOR_2SM), i8.last_path()
+    H.assert_same(got, want, p.name)
+    H.not_degenerate(want)
 
 
 @pytest.mark.parametrize("batch,M,N,K", [(2, 64, 64, 64), (7, 64, 64, 64), (1, 64, 64, 64), (6, 64, 32, 64), (5, 17, 64, 48),
