@@ -165,20 +165,6 @@ __device__ __forceinline__ void epilogue_chunk_shift32(const int32_t (&v)[32], c
     }
 }
 
-// Folded form: the bias rides in the 64-bit addend, ReLU is applied to the packed bytes (needs m2 >= 0 under ReLU).
-template <bool RELU>
-__device__ __forceinline__ void epilogue_chunk_fold(const int32_t (&v)[32], const int32_t* s_m2, const long long* s_c64, int c0,
-                                                    uint32_t (&out)[8]) {
-#pragma unroll
-    for (int j = 0; j < 8; j++) {
-        const int4 m2 = *reinterpret_cast<const int4*>(s_m2 + c0 + 4 * j);
-        const longlong2 ca = *reinterpret_cast<const longlong2*>(s_c64 + c0 + 4 * j);
-        const longlong2 cb = *reinterpret_cast<const longlong2*>(s_c64 + c0 + 4 * j + 2);
-        const uint32_t pk = pack_sat4(requant_fold(v[4 * j + 0], m2.x, ca.x), requant_fold(v[4 * j + 1], m2.y, ca.y),
-                                      requant_fold(v[4 * j + 2], m2.z, cb.x), requant_fold(v[4 * j + 3], m2.w, cb.y));
-        out[j] = RELU ? relu_s8x4(pk) : pk;
-    }
-}
 // Folded form with the bias added explicitly: two words per channel from shared memory instead of three (a 16-byte
 // shared-memory broadcast costs four wavefronts, and eight epilogue warps each fetch every channel's constants).
 template <bool RELU>
