@@ -227,6 +227,8 @@ typedef struct {
     int waves;           /* ceil(tiles / workers) */
     int b_resident;      /* B fetched once per CTA and kept in shared memory */
     int epilogue_warps;
+    int kernel;          /* 0: large-tile kernel (rows of C on the tensor-memory lanes); 1: channel-major kernel: tile_m is
+                            then the strip of rows per tile (a multiple of 16) and tile_n the channel block, 128 or 256 */
 } i8_plan;
 
 /* Fills *out with the plan gemm_i8 would launch for K-contiguous operands of shape (M, N, K) on a device with sm_count

@@ -236,7 +236,7 @@ def mpc_forward_f32(Adyn, Bdyn, Kinf, x0, d, u, xs=None, stream=None) -> None:
 
 class Plan(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("shape_class", "tile_m", "tile_n", "stages", "cta_group", "raster_group", "sticky",
-                                             "m_tiles", "n_tiles", "workers", "waves", "b_resident", "epilogue_warps")]
+                                             "m_tiles", "n_tiles", "workers", "waves", "b_resident", "epilogue_warps", "kernel")]
 
 
 def plan_gemm(M: int, N: int, K: int, sm_count: int = 148) -> dict:

@@ -351,7 +351,8 @@ struct TcPlan {
     int b_resident;
     int shape_cls;
 };
-static thread_local TcPlan t_last_plan = {};
+static thread_local i8_plan t_last_plan = {};     // what the last launch of a tensor kernel by this thread used
+static void fill_plan(const TcPlan& pl, i8_plan* out);
 
 // CTA pairs: their larger tiles and cluster set-up cost about 1.5 us more per launch, which pays once there is at least
 // one full wave of 256-row tiles and enough K per cluster (measured crossover: waves x K blocks ~ 48).
@@ -424,7 +425,7 @@ static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap
     const bool two_sm = pl.two_sm != 0;
     const int bn = pl.bn;
     const int b_rows = two_sm ? bn / 2 : bn;           // rows of the B tile one CTA loads
-    t_last_plan = pl;
+    fill_plan(pl, &t_last_plan);
     t_used_two_sm = two_sm;
     CUtensorMap tmB;
     if (kl.b_mn) {
@@ -545,6 +546,40 @@ struct SwapPlan {
     int off_b, off_bar, smem_bytes;
     double cycles;             // the cost model's estimate for the whole launch
 };
+static void fill_plan_swap(const SwapPlan& sp, int M, int N, i8_plan* out) {
+    out->shape_class = shape_class(M, N);
+    out->kernel = 1;
+    out->tile_m = sp.pw;                        // rows of C per tile: the strip
+    out->tile_n = sp.two_sm ? 256 : 128;        // columns of C per tile: the channel block
+    out->stages = sp.stages;
+    out->cta_group = sp.two_sm ? 2 : 1;
+    out->raster_group = 0;
+    out->sticky = 0;
+    out->m_tiles = sp.m_tiles;
+    out->n_tiles = sp.n_blocks;
+    out->workers = sp.workers;
+    out->waves = sp.workers ? (sp.num_tiles + sp.workers - 1) / sp.workers : 0;
+    out->b_resident = 0;
+    out->epilogue_warps = SWAP_EPI_WARPS;
+}
+
+static void fill_plan(const TcPlan& pl, i8_plan* out) {
+    out->shape_class = pl.shape_cls;
+    out->kernel = 0;
+    out->tile_m = pl.tile_m;
+    out->tile_n = pl.bn;
+    out->stages = pl.stages;
+    out->cta_group = pl.two_sm ? 2 : 1;
+    out->raster_group = pl.group_m;
+    out->sticky = pl.sticky;
+    out->m_tiles = pl.m_tiles;
+    out->n_tiles = pl.n_tiles;
+    out->workers = pl.workers;
+    out->waves = pl.workers ? (pl.num_tiles + pl.workers - 1) / pl.workers : 0;
+    out->b_resident = pl.b_resident;
+    out->epilogue_warps = 8;
+}
+
 
 // Strip width: every candidate (multiples of 16) is priced as waves x (ring slots per tile x cycles per slot + a fixed
 // cost per tile) + the exposed read-out of the last tile.  A slot's cycles are the larger of its four instructions
@@ -631,6 +666,7 @@ static int run_swap(DeviceCtx* ctx, bool conv, const SwapPlan& pl, const CUtenso
     p.wait_limit_cycles = (long long)(g_wait_limit_ns * 2);
     p.dev_status = ctx->dev_status;
     t_used_two_sm = pl.two_sm != 0;
+    fill_plan_swap(pl, M, N, &t_last_plan);
     if (conv) return pl.two_sm ? launch_swap<true, true>(ctx, 21, pl, tmW, tmX, p, st) : launch_swap<true, false>(ctx, 22, pl, tmW, tmX, p, st);
     return pl.two_sm ? launch_swap<false, true>(ctx, 23, pl, tmW, tmX, p, st) : launch_swap<false, false>(ctx, 24, pl, tmW, tmX, p, st);
 }
@@ -1206,33 +1242,21 @@ int mpc_forward_f32(const float* Adyn, const float* Bdyn, const float* Kinf, con
     return I8_OK;
 }
 
-static void fill_plan(const TcPlan& pl, i8_plan* out) {
-    out->shape_class = pl.shape_cls;
-    out->tile_m = pl.tile_m;
-    out->tile_n = pl.bn;
-    out->stages = pl.stages;
-    out->cta_group = pl.two_sm ? 2 : 1;
-    out->raster_group = pl.group_m;
-    out->sticky = pl.sticky;
-    out->m_tiles = pl.m_tiles;
-    out->n_tiles = pl.n_tiles;
-    out->workers = pl.workers;
-    out->waves = pl.workers ? (pl.num_tiles + pl.workers - 1) / pl.workers : 0;
-    out->b_resident = pl.b_resident;
-    out->epilogue_warps = 8;
-}
-
 int i8ops_plan_gemm(int M, int N, int K, int sm_count, i8_plan* out) {
     if (!out) return I8_ERR_NULL;
     if (M <= 0 || N <= 0 || K <= 0 || sm_count <= 0) return I8_ERR_SHAPE;
     const KLoop kl = gemm_kloop(K);
+    if (swap_wanted(false, M, N, K, kl.num_kblocks, kl.num_iters, kl.num_kblocks, BK, sm_count)) {
+        const SwapPlan sp = plan_swap(M, N, kl.num_iters, N > 128, sm_count);
+        if (sp.pw && sp.stages >= 2) { fill_plan_swap(sp, M, N, out); return I8_OK; }
+    }
     fill_plan(plan_tc(false, M, N, K, kl.num_kblocks, kl.num_iters, kl.num_kblocks, BK, sm_count), out);
     return I8_OK;
 }
 
 int i8ops_last_plan(i8_plan* out) {
     if (!out) return I8_ERR_NULL;
-    fill_plan(t_last_plan, out);
+    *out = t_last_plan;
     return I8_OK;
 }
 

@@ -58,6 +58,23 @@ def test_gemm_argument_validation(L):
     assert L.i8ops_last_path() == 0
 
 
+def test_float_scale_and_probe_argument_validation(L):
+    P = ctypes.c_void_p
+    buf = (ctypes.c_int8 * 4096)()
+    f32 = (ctypes.c_float * 64)()
+    a = P(ctypes.addressof(buf)); q = P(ctypes.addressof(f32))
+
+    def call(A=a, B=a, C=a, scale=q, M=16, N=16, K=16, a_rs=16, b_cs=16, ldc=16):
+        return L.gemm_i8_fscale(A, a_rs, 1, B, 1, b_cs, C, ldc, None, scale, 0, M, N, K, 0, None)
+    assert call(scale=None) == 1 and call(A=None) == 1 and call(C=None) == 1          # I8_ERR_NULL
+    assert call(M=-1) == 2 and call(K=65537) == 5 and call(ldc=8) == 3 and call(a_rs=8) == 3
+    assert call(M=0) == 0 and call(N=0) == 0
+    # the issue-rate probe checks its ranges before any CUDA call
+    assert L.i8ops_probe_mma_rate(256, 4096, 1, None, None) == 1
+    for bad in ((8, 4096, 1), (272, 4096, 1), (250, 4096, 1), (256, 100, 1), (256, 32, 1), (256, 4096, 0)):
+        assert L.i8ops_probe_mma_rate(bad[0], bad[1], bad[2], a, None) == 5, bad
+
+
 def test_batched_and_conv_argument_validation(L):
     P = ctypes.c_void_p
     buf = (ctypes.c_int8 * 4096)()

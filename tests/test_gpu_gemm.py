@@ -329,6 +329,13 @@ def test_recorded_class_plan_runs_and_is_reported():
         H.assert_same(got, H.gemm_oracle(p), p.name)
     finally:
         i8.set_class_plan(0, base=(8192, 8192, 8192), tile_n=256, cta_group=2, raster_group=16)
+    # a shape the occupancy rule sends to the channel-major kernel: 12544 x 256 x 1152 (98 large tiles on 148 SMs)
+    p = inputs.make_gemm(12544, 256, 1152, 4150, per_channel=1, relu=1)
+    got = H.gemm_gpu(p)
+    ran, asked = i8.last_plan(), i8.plan_gemm(p.M, p.N, p.K)
+    assert i8.last_path() == i8.PATH_CHANNEL_MAJOR_2SM and ran["kernel"] == 1 and ran == asked
+    assert ran["tile_n"] == 256 and ran["tile_m"] % 16 == 0 and ran["m_tiles"] * ran["tile_m"] >= p.M and ran["workers"] <= 74
+    H.assert_same(got, H.gemm_oracle(p), p.name)
     # without a recorded entry nearby, what ran is still what the query reports (config 1a: CTA pairs by the rule)
     p = inputs.make_gemm(2048, 2304, 1024, 4200, per_channel=1, relu=0)
     got = H.gemm_gpu(p)
