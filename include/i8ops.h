@@ -141,6 +141,11 @@ int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs,
  *   x  device int8 [N][H][W][C] (NHWC, dense);  w  device int8 [K][R][S][C] (dense);
  *   y  device int8 [N][P][Q][K] (dense),  P = floor((H + 2*pad_h - R)/stride_h) + 1, Q likewise.
  *   bias/mult/shift indexed by filter k.
+ * Layers that the implicit-GEMM loads do not take (an activation tensor below 128 KiB, a stride above 8, a filter side or
+ * padding above 16) run, when C % 16 == 0, as an unfold pass into the GEMM form's A matrix followed by the tensor GEMM;
+ * that matrix (N*P*Q x R*S*C bytes, at most 256 MiB) is allocated and released in stream order from a memory pool the
+ * library keeps per device, so the call stays asynchronous and may be captured into a CUDA graph.
+ * i8ops_last_conv_unfolded() tells whether the most recent convolution of this thread ran that way.
  * Errors: I8_ERR_NULL, I8_ERR_SHAPE (a non-positive extent or an empty output), I8_ERR_UNSUPPORTED
  * (stride < 1, pad < 0), I8_ERR_RANGE (R*S*C > 65536), I8_ERR_CUDA.
  */
@@ -148,6 +153,8 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y,
               const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel,
               int N, int H, int W, int C, int K, int R, int S,
               int stride_h, int stride_w, int pad_h, int pad_w, int relu, void* stream);
+
+int i8ops_last_conv_unfolded(void);
 
 /*
  * Host-buffer variants: every pointer is HOST memory (pinned memory makes the copies asynchronous).

@@ -43,6 +43,7 @@ SIGNATURES = {
     "i8ops_probe_mma_rate": (_int, [_int, _int, _int, _vp, _vp]),
     "i8ops_last_cuda_error": (_int, []),
     "i8ops_last_path": (_int, []),
+    "i8ops_last_conv_unfolded": (_int, []),
     "i8ops_set_path": (_int, [_int]),
     "i8ops_set_wait_limit_ms": (None, [_int]),
     "i8ops_version": (_int, []),
@@ -262,6 +263,11 @@ def set_class_plan(shape_class: int, base=(0, 0, 0), tile_n: int = 0, cta_group:
     """Record a schedule for a shape class (see ``i8ops_set_class_plan``); all defaults forgets the entry."""
     _check(lib().i8ops_set_class_plan(int(shape_class), int(base[0]), int(base[1]), int(base[2]), int(tile_n), int(cta_group),
                                       int(raster_group), int(sticky)), "i8ops_set_class_plan")
+
+
+def last_conv_unfolded() -> bool:
+    """Whether the calling thread's most recent convolution ran as an unfold pass followed by the tensor GEMM."""
+    return bool(lib().i8ops_last_conv_unfolded())
 
 
 def tmap_cache_stats():

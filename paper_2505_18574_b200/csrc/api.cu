@@ -36,6 +36,8 @@ struct DeviceCtx {
     cudaStream_t s_in = nullptr, s_out = nullptr;   // copy streams of the host-buffer variants
     cudaEvent_t ev[2 * 8 + 2] = {};                 // chunk hand-over events (up to 8 row chunks)
     std::mutex host_mutex;                          // serialises the host-buffer variant: its calls share ws, s_in, s_out and ev
+    std::atomic<bool> pool_ready{false};            // stream-ordered pool of the unfolded-convolution workspaces (made on first use)
+    cudaMemPool_t pool = nullptr;
 };
 
 static DeviceCtx g_ctx[MAX_DEVICES];
@@ -53,11 +55,13 @@ static int g_swap = 1;                           // channel-major kernel: 0 neve
 static int g_swap_stages = 0;                    // ring slots of the channel-major kernel: 0 = as many as fit (I8OPS_SWAP_STAGES)
 static int g_swap_pw = 0;                        // strip width override for tuning (I8OPS_SWAP_PW)
 static int g_slab = 1;                           // slab-resident stride-1 convolution kernel (I8OPS_SLAB=0 turns it off)
+static int g_unfold = 1;                         // unfold + tensor GEMM for convolutions the im2col maps do not take (I8OPS_UNFOLD=0 turns it off)
 
 static thread_local int t_last_path = I8_PATH_NONE;
 static thread_local int t_last_cuda = 0;
 static thread_local bool t_used_two_sm = false;
 static thread_local bool t_used_swap = false;     // the last tensor-path launch was the channel-major kernel
+static thread_local bool t_last_unfold = false;   // the last convolution ran as unfold + tensor GEMM
 static thread_local bool t_tmap_failed = false;   // the last tensor-path attempt stopped at a tensor-map encoding (nothing launched)
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -120,6 +124,8 @@ static int get_ctx(DeviceCtx** out) {
         if (sticky) g_sticky = atoi(sticky);
         const char* slab = getenv("I8OPS_SLAB");
         if (slab) g_slab = atoi(slab);
+        const char* unf = getenv("I8OPS_UNFOLD");
+        if (unf) g_unfold = atoi(unf);
         const char* sw = getenv("I8OPS_SWAP");
         if (sw) g_swap = atoi(sw);
         const char* sws = getenv("I8OPS_SWAP_STAGES");
@@ -745,6 +751,50 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     return run_tc(ctx, true, pl, tmA, kl, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
 }
 
+// Convolutions the im2col tensor maps do not take (small activation tensors, long strides, large filters) with
+// C % 16 == 0: the activations are unfolded into the GEMM form's A matrix in a workspace that lives in stream order
+// (allocated from the library's own pool before the two launches and released behind them, so concurrent streams never
+// share it and a captured graph owns its copy), then the product runs on the tensor path.  Returns I8_ERR_UNSUPPORTED,
+// launching nothing, when the workspace would be too large or cannot be had.
+static const int64_t UNFOLD_MAX_BYTES = 256ll << 20;
+static int run_conv_unfold(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, const int32_t* mult,
+                           const int32_t* shift, int per_channel, int N, int H, int W, int C, int Kf, int R, int S, int P, int Q,
+                           int stride_h, int stride_w, int pad_h, int pad_w, int relu, cudaStream_t st) {
+    const int64_t M = (int64_t)N * P * Q, K = (int64_t)R * S * C;
+    if (C % 16 != 0 || M >= (1ll << 31) || M * K > UNFOLD_MAX_BYTES) return I8_ERR_UNSUPPORTED;
+    if (!ctx->pool_ready.load(std::memory_order_acquire)) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!ctx->pool_ready.load(std::memory_order_relaxed)) {
+            int dev = 0;
+            CUDA_TRY(cudaGetDevice(&dev));
+            cudaMemPoolProps props{};
+            props.allocType = cudaMemAllocationTypePinned;
+            props.handleTypes = cudaMemHandleTypeNone;
+            props.location.type = cudaMemLocationTypeDevice;
+            props.location.id = dev;
+            if (cudaMemPoolCreate(&ctx->pool, &props) != cudaSuccess) { cudaGetLastError(); return I8_ERR_UNSUPPORTED; }
+            uint64_t keep = ~0ull;                  // released blocks stay in the pool: the next call reuses them
+            cudaMemPoolSetAttribute(ctx->pool, cudaMemPoolAttrReleaseThreshold, &keep);
+            ctx->pool_ready.store(true, std::memory_order_release);
+        }
+    }
+    void* a = nullptr;
+    if (cudaMallocFromPoolAsync(&a, (size_t)(M * K), ctx->pool, st) != cudaSuccess) { cudaGetLastError(); return I8_ERR_UNSUPPORTED; }
+    UnfoldParams u{x, (int8_t*)a, N, H, W, C, R, S, P, Q, stride_h, stride_w, pad_h, pad_w};
+    const int64_t pieces = M * K / 16;
+    int64_t blocks = (pieces + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    conv_unfold_i8_kernel<<<(int)blocks, 256, 0, st>>>(u);
+    const cudaError_t le = cudaGetLastError();
+    int rc = le == cudaSuccess ? I8_OK : cuda_fail(le);
+    if (rc == I8_OK) {
+        t_used_two_sm = false; t_tmap_failed = false;
+        rc = run_gemm_tc(ctx, (const int8_t*)a, K, w, K, y, Kf, bias, mult, shift, per_channel, (int)M, Kf, (int)K, relu, st);
+    }
+    cudaFreeAsync(a, st);
+    return rc;
+}
+
 // Slab-resident stride-1 convolution (conv_slab.cuh): plan and launch.  Returns I8_ERR_UNSUPPORTED, launching nothing,
 // when the layer does not fit the kernel (the caller then takes the implicit-GEMM path).
 static int run_conv_slab(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, const int32_t* mult,
@@ -1033,6 +1083,7 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
               int per_channel, int N, int H, int W, int C, int K, int R, int S, int stride_h, int stride_w, int pad_h,
               int pad_w, int relu, void* stream) {
     t_last_path = I8_PATH_NONE;
+    t_last_unfold = false;
     if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || K <= 0 || R <= 0 || S <= 0) return I8_ERR_SHAPE;
     if (stride_h < 1 || stride_w < 1 || pad_h < 0 || pad_w < 0) return I8_ERR_UNSUPPORTED;
     if (H + 2 * pad_h < R || W + 2 * pad_w < S) return I8_ERR_SHAPE;
@@ -1072,6 +1123,12 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
             if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
     }
+    if (g_path_mode != 1 && g_unfold && aligned16(x) && aligned16(w)) {
+        rc = run_conv_unfold(ctx, x, w, y, bias, mult, shift, per_channel, N, H, W, C, K, R, S, P, Q, stride_h, stride_w,
+                             pad_h, pad_w, relu, st);
+        if (rc == I8_OK) { t_last_path = tensor_path_used(); t_last_unfold = true; return rc; }
+        if (rc != I8_ERR_UNSUPPORTED && !(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
+    }
     GenericConvParams g{x, w, y, bias, mult, shift, per_channel, relu, N, H, W, C, K, R, S, P, Q, stride_h, stride_w, pad_h, pad_w};
     const int64_t total = (int64_t)N * P * Q * K;
     int64_t blocks = (total + 255) / 256;
@@ -1081,6 +1138,8 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
     t_last_path = I8_PATH_GENERIC;
     return I8_OK;
 }
+
+int i8ops_last_conv_unfolded(void) { return t_last_unfold ? 1 : 0; }
 
 int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C, const int32_t* bias, const int32_t* mult, const int32_t* shift,
                  int per_channel, int M, int N, int K, int relu, void* stream) {

@@ -78,6 +78,33 @@ __global__ void __launch_bounds__(256) conv2d_i8_generic_kernel(const GenericCon
     }
 }
 
+// Unfolds NHWC activations into the row-major matrix [N*P*Q][R*S*C] of the convolution's GEMM form (the column order
+// (r, s, c) of the KRSC filters), zeros where a tap falls into the padding.  One 16-byte piece per thread and step
+// (C % 16 == 0).  Used for the layers the im2col tensor maps do not take; the product then runs on the tensor path.
+struct UnfoldParams {
+    const int8_t* x; int8_t* a;
+    int N, H, W, C, R, S, P, Q, stride_h, stride_w, pad_h, pad_w;
+};
+
+__global__ void __launch_bounds__(256) conv_unfold_i8_kernel(const UnfoldParams p) {
+    const int c16 = p.C >> 4;
+    const int64_t total = (int64_t)p.N * p.P * p.Q * p.R * p.S * c16;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % c16);
+        int64_t rest = idx / c16;
+        const int s = (int)(rest % p.S); rest /= p.S;
+        const int r = (int)(rest % p.R); rest /= p.R;
+        const int q = (int)(rest % p.Q); rest /= p.Q;
+        const int pp = (int)(rest % p.P);
+        const int n = (int)(rest / p.P);
+        const int h = pp * p.stride_h - p.pad_h + r, ww = q * p.stride_w - p.pad_w + s;
+        int4 v = make_int4(0, 0, 0, 0);
+        if (h >= 0 && h < p.H && ww >= 0 && ww < p.W)
+            v = __ldg(reinterpret_cast<const int4*>(p.x + (((int64_t)n * p.H + h) * p.W + ww) * p.C) + c);
+        reinterpret_cast<int4*>(p.a)[idx] = v;     // idx is exactly the piece's position in the unfolded matrix
+    }
+}
+
 // Self-test of the bounded wait: one CTA waits on an mbarrier that nothing ever signals.  The wait must give
 // up after `limit_cycles`, record DEV_TIMEOUT_TEST in the status word and return normally.
 __global__ void bounded_wait_selftest_kernel(long long limit_cycles, unsigned* dev_status) {

@@ -81,6 +81,73 @@ def test_conv_cta_pair_kernel(N, H_, W, C, K, R, S, st, pad):
     H.assert_same(got, want, p.name + " two-SM")
 
 
+@pytest.mark.parametrize("N,H_,W,C,K,R,S,st,pad", [
+    (1, 7, 7, 512, 512, 3, 3, 1, 1),      # the last ResNet-50 stage at batch 1: 25 KB of activations
+    (1, 14, 14, 256, 256, 3, 3, 2, 1),    # stride 2, 50 KB
+    (2, 9, 9, 48, 40, 5, 5, 3, 2),        # channels a multiple of 16 only, ragged filter count
+    (1, 28, 28, 128, 160, 3, 3, 1, 0),    # 100 KB, no padding, several row tiles, too many filters for the slab kernel
+    (4, 40, 40, 32, 64, 3, 3, 9, 1),      # a stride beyond the im2col loads' range on a large tensor
+    (1, 20, 21, 16, 32, 17, 3, 1, 8),     # a filter side beyond the im2col loads' range
+    (3, 5, 6, 16, 8, 2, 4, 1, 3),         # tiny: padding wider than the image's half
+])
+def test_conv_unfolded_layers_take_the_tensor_path(N, H_, W, C, K, R, S, st, pad):
+    """Layers outside the im2col loads' reach (small activation tensors, long strides, large filters) with C % 16 == 0:
+    unfold pass + tensor GEMM, bit-exact against the oracle; the generic kernel when the unfold path is ruled out."""
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_conv(N, H_, W, C, K, R, S, st, pad, 1300 + N + H_ + C + K)
+    want = H.conv_oracle(p)
+    got = H.conv_gpu(p)
+    assert i8.last_conv_unfolded(), p.name
+    assert i8.last_path() in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM, i8.PATH_CHANNEL_MAJOR, i8.PATH_CHANNEL_MAJOR_2SM), i8.last_path()
+    H.assert_same(got, want, p.name + " unfolded")
+    H.assert_same(H.conv_gpu(p), want, p.name + " unfolded, second call (workspace reused from the pool)")
+    i8.set_path(1)
+    H.assert_same(H.conv_gpu(p), want, p.name + " generic")
+    assert not i8.last_conv_unfolded() and i8.last_path() == i8.PATH_GENERIC
+
+
+def test_conv_unfolded_inside_a_cuda_graph_and_on_two_streams():
+    """The unfold workspace lives in stream order: a captured graph owns its copy (replays give the same bytes), and two
+    streams running different layers at once do not share it."""
+    import torch
+    import paper_2505_18574_b200 as i8
+    dev = torch.device("cuda", 0)
+    ps = [inputs.make_conv(1, 14, 14, 256, 256, 3, 3, 1, 1, 1401), inputs.make_conv(1, 7, 7, 512, 384, 3, 3, 1, 1, 1402)]
+    wants = [H.conv_oracle(p) for p in ps]
+
+    def dev_args(p):
+        T = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+        y = torch.zeros((p.N, p.P, p.Q, p.K), dtype=torch.int8, device=dev)
+        return (T(p.x), T(p.w), y, T(p.bias), T(p.mult), T(p.shift), p.per_channel, p.relu, (p.stride_h, p.stride_w), (p.pad_h, p.pad_w))
+
+    args = [dev_args(p) for p in ps]
+    # two streams, interleaved launches
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for _ in range(8):
+        for a, s in zip(args, streams):
+            with torch.cuda.stream(s):
+                i8.conv2d_i8(*a)
+                assert i8.last_conv_unfolded()
+    torch.cuda.synchronize()
+    for a, w, p in zip(args, wants, ps):
+        H.assert_same(a[2].cpu().numpy(), w, p.name + " two streams")
+        a[2].zero_()
+    # graph capture and three replays
+    g = torch.cuda.CUDAGraph(); s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            for a in args:
+                i8.conv2d_i8(*a)
+    for _ in range(3):
+        for a in args:
+            a[2].zero_()
+        g.replay(); torch.cuda.synchronize()
+        for a, w, p in zip(args, wants, ps):
+            H.assert_same(a[2].cpu().numpy(), w, p.name + " graph replay")
+    assert i8.last_device_status() == 0
+
+
 def test_conv_delta_filter_on_gpu():
     """Oracle-independent: a filter with a single 1 copies a shifted view of the input."""
     import paper_2505_18574_b200 as i8
