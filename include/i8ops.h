@@ -145,6 +145,7 @@ int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs,
  * padding above 16) run, when C % 16 == 0, as an unfold pass into the GEMM form's A matrix followed by the tensor GEMM;
  * that matrix (N*P*Q x R*S*C bytes, at most 256 MiB) is allocated and released in stream order from a memory pool the
  * library keeps per device, so the call stays asynchronous and may be captured into a CUDA graph.
+ * The first such call on a device creates the pool: make it outside any stream capture.
  * i8ops_last_conv_unfolded() tells whether the most recent convolution of this thread ran that way.
  * Errors: I8_ERR_NULL, I8_ERR_SHAPE (a non-positive extent or an empty output), I8_ERR_UNSUPPORTED
  * (stride < 1, pad < 0), I8_ERR_RANGE (R*S*C > 65536), I8_ERR_CUDA.
@@ -213,7 +214,11 @@ int i8ops_last_device_status(void* stream);
  *   x0 [batch][12], d [batch][nhorizon][4]      device, fp32, 16-byte aligned
  *   u  [batch][nhorizon][4]                     device output, fp32, 16-byte aligned
  *   xs [batch][nhorizon][12] or NULL            device output: the states x[0..nhorizon-1]
- * Arithmetic is fp32 with fused multiply-adds in ascending index order (the paper's precision).
+ * Arithmetic is fp32 with fused multiply-adds in ascending index order (the paper's precision; two output rows share
+ * one packed instruction, each half rounded as the scalar instruction would).
+ * Without xs and for horizons up to 12 steps, persistent CTAs stream chunks of 128 instances through a shared-memory ring
+ * (bulk copies in, bulk copies out; every wait bounded, see i8ops_last_device_status); otherwise one thread per
+ * instance loads and stores its own records.  Same arithmetic, same results.
  * Errors: I8_ERR_SHAPE (negative batch or nhorizon), I8_ERR_NULL, I8_ERR_ALIGN, I8_ERR_CUDA.
  */
 int mpc_forward_f32(const float* Adyn, const float* Bdyn, const float* Kinf, const float* x0, const float* d, float* u,

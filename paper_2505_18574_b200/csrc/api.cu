@@ -55,6 +55,7 @@ static int g_swap = 1;                           // channel-major kernel: 0 neve
 static int g_swap_stages = 0;                    // ring slots of the channel-major kernel: 0 = as many as fit (I8OPS_SWAP_STAGES)
 static int g_swap_pw = 0;                        // strip width override for tuning (I8OPS_SWAP_PW)
 static int g_slab = 1;                           // slab-resident stride-1 convolution kernel (I8OPS_SLAB=0 turns it off)
+static int g_mpc_stream = 1;                     // streaming TinyMPC kernel: 0 off, 1 on, 2..4 ring slots (I8OPS_MPC_STREAM)
 static int g_unfold = 1;                         // unfold + tensor GEMM for convolutions the im2col maps do not take (I8OPS_UNFOLD=0 turns it off)
 
 static thread_local int t_last_path = I8_PATH_NONE;
@@ -124,6 +125,8 @@ static int get_ctx(DeviceCtx** out) {
         if (sticky) g_sticky = atoi(sticky);
         const char* slab = getenv("I8OPS_SLAB");
         if (slab) g_slab = atoi(slab);
+        const char* mps = getenv("I8OPS_MPC_STREAM");
+        if (mps) g_mpc_stream = atoi(mps);
         const char* unf = getenv("I8OPS_UNFOLD");
         if (unf) g_unfold = atoi(unf);
         const char* sw = getenv("I8OPS_SWAP");
@@ -1289,12 +1292,49 @@ int mpc_forward_f32(const float* Adyn, const float* Bdyn, const float* Kinf, con
     int rc = get_ctx(&ctx);
     if (rc) return rc;
     MpcMatrices m;
-    memcpy(m.A, Adyn, sizeof(m.A));
-    memcpy(m.B, Bdyn, sizeof(m.B));
-    memcpy(m.K, Kinf, sizeof(m.K));
+    for (int r = 0; r < MPC_NX; r++) {
+        for (int c = 0; c < MPC_NX; c++) m.At[c][r] = Adyn[r * MPC_NX + c];
+        for (int c = 0; c < MPC_NU; c++) m.Bt[c][r] = Bdyn[r * MPC_NU + c];
+    }
+    for (int r = 0; r < MPC_NU; r++)
+        for (int c = 0; c < MPC_NX; c++) m.Kt[c][r] = -Kinf[r * MPC_NX + c];
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!xs && g_mpc_stream && (int64_t)batch * nhorizon < (1ll << 27)) {
+        // streaming kernel: chunks of 256 instances (128 for longer horizons) while two ring slots fit in 72 KB; beyond
+        // that the direct kernel
+        const int64_t per_inst = MPC_NX * 4 + 16 * (int64_t)nhorizon, tail = MPC_MAX_STAGES * 8 + 16, budget = 72 * 1024;
+        const int stages = g_mpc_stream >= 2 && g_mpc_stream <= MPC_MAX_STAGES ? g_mpc_stream : 2;
+        const int chunk = stages * 256 * per_inst + tail <= budget ? 256 : (stages * 128 * per_inst + tail <= budget ? 128 : 0);
+        if (chunk) {
+            const int smem = (int)(stages * chunk * per_inst + tail);
+            auto kern = chunk == 256 ? mpc_forward_stream_kernel<256> : mpc_forward_stream_kernel<128>;
+            const int slot = chunk == 256 ? 25 : 26;
+            if (!ctx->attr_set[slot]) {
+                CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+                ctx->attr_set[slot] = true;
+            }
+            static thread_local int occ_key = -1, occ_val = 0;    // resident CTAs per SM for (chunk, shared memory)
+            if (occ_key != chunk * 1000003 + smem) {
+                CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_val, kern, chunk, smem));
+                occ_key = chunk * 1000003 + smem;
+            }
+            const int64_t chunks = ((int64_t)batch + chunk - 1) / chunk;
+            // Measured optimum: 384-512 resident threads per SM (2^20 instances, horizon 5: 57 / 45.4 / 53 us with one / two /
+            // three CTAs of 256 threads, 57 / 46.5 / 49 / 56 us with two / three / four / six CTAs of 128): fewer leave the
+            // fp32 pipe's latency exposed, more slow the memory side down.
+            const int want = chunk == 256 ? 2 : 3;
+            const int per_sm = occ_val < 1 ? 1 : (occ_val < want ? occ_val : want);
+            int64_t blocks = (int64_t)ctx->sm_count * per_sm;
+            if (blocks > chunks) blocks = chunks;
+            MpcStreamParams sp{x0, d, u, batch, nhorizon, stages, (long long)(g_wait_limit_ns * 2), ctx->dev_status};
+            kern<<<(int)blocks, chunk, smem, st>>>(m, sp);
+            CUDA_TRY(cudaGetLastError());
+            t_last_path = I8_PATH_GENERIC;
+            return I8_OK;
+        }
+    }
     int blocks = (batch + 127) / 128;
     if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
-    cudaStream_t st = (cudaStream_t)stream;
     mpc_forward_f32_kernel<<<blocks, 128, 0, st>>>(m, (const float4*)x0, (const float4*)d, (float4*)u, (float4*)xs, batch, nhorizon);
     CUDA_TRY(cudaGetLastError());
     t_last_path = I8_PATH_GENERIC;

@@ -26,7 +26,10 @@ def _run(p, states=False):
     return u.cpu().numpy(), (xs.cpu().numpy() if states else None)
 
 
-@pytest.mark.parametrize("batch,nh", [(1, 5), (7, 5), (256, 5), (1000, 1), (4099, 8), (100000, 5), (129, 9), (3000, 12)])
+# horizons up to 5 stream chunks of 256 instances, up to 14 chunks of 128, longer ones take one thread per instance;
+# 300000 and 700001 instances give every persistent CTA several rounds (ring slots refilled, barrier phases flipping)
+@pytest.mark.parametrize("batch,nh", [(1, 5), (7, 5), (256, 5), (1000, 1), (4099, 8), (100000, 5), (129, 9), (3000, 12),
+                                      (300000, 5), (700001, 3), (150000, 14), (2000, 20), (257, 5), (255, 2)])
 def test_mpc_forward_matches_oracle(batch, nh):
     import oracle
     p = inputs.make_mpc(batch, nh, seed=40 + nh)
