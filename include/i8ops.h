@@ -298,7 +298,9 @@ int i8ops_last_path(void);
 /* Restrict dispatch: 0 = automatic (default), 1 = always the generic kernel, 2 = GEMMs and convolutions take the
  * two-SM tensor kernel whenever the layout allows the tensor path (also where its large tiles do not pay),
  * 3 = automatic among the large-tile kernels only (no slab kernel, no channel-major kernel),
- * 4 = GEMMs and implicit-GEMM convolutions take the channel-major kernel whenever the layout allows the tensor path.
+ * 4 = GEMMs and implicit-GEMM convolutions take the channel-major kernel whenever the layout allows the tensor path
+ *     (single CTAs or CTA pairs by its cost model), 5 = the same on CTA pairs whenever there are more than 128 channels,
+ *     6 = the same on single CTAs only.
  * Returns the previous setting. */
 int i8ops_set_path(int mode);
 

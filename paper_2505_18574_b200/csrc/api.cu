@@ -52,6 +52,7 @@ static int g_tma_store = 1;                      // read-out of the wide tiles t
 static int g_sticky = 1;                         // column-sticky tile order for short-K problems (I8OPS_STICKY=0 turns it off)
 static int g_tmap_cache = 1;                     // per-thread cache of encoded tensor maps (I8OPS_TMAP_CACHE=0 encodes every time)
 static int g_swap = 1;                           // channel-major kernel: 0 never, 1 by rule, 2 wherever legal (I8OPS_SWAP)
+static int g_swap_two_sm = -1;                   // channel-major kernel on CTA pairs: -1 by cost, 0 never, 1 whenever N > 128 (I8OPS_SWAP_2SM)
 static int g_swap_stages = 0;                    // ring slots of the channel-major kernel: 0 = as many as fit (I8OPS_SWAP_STAGES)
 static int g_swap_pw = 0;                        // strip width override for tuning (I8OPS_SWAP_PW)
 static int g_slab = 1;                           // slab-resident stride-1 convolution kernel (I8OPS_SLAB=0 turns it off)
@@ -131,6 +132,8 @@ static int get_ctx(DeviceCtx** out) {
         if (unf) g_unfold = atoi(unf);
         const char* sw = getenv("I8OPS_SWAP");
         if (sw) g_swap = atoi(sw);
+        const char* sw2 = getenv("I8OPS_SWAP_2SM");
+        if (sw2) g_swap_two_sm = atoi(sw2);
         const char* sws = getenv("I8OPS_SWAP_STAGES");
         if (sws) g_swap_stages = atoi(sws);
         const char* swp = getenv("I8OPS_SWAP_PW");
@@ -634,6 +637,19 @@ static SwapPlan plan_swap(int M, int N, int num_iters, bool two_sm, int sm_count
     return best;
 }
 
+// CTA pairs halve the activation bytes each CTA pulls from L2 but cost a fixed amount per launch (cluster scheduling,
+// two cluster barriers, the paired commit): on the 12544 x 256 x 1152 / 2304 convolutions the model's 1270- / 2540-cycle
+// advantage for pairs is a 0.63 / 0.55 us loss in fact (8.37 -> 7.72 and 10.2 -> 9.65 us on single CTAs), i.e. 2300-3500
+// cycles.  Pairs are taken only where the model still sees them ahead by more than that.
+static const double SWAP_PAIR_FIXED_CYCLES = 4000.0;
+static SwapPlan plan_swap_auto(int M, int N, int num_iters, int sm_count) {
+    const SwapPlan one = plan_swap(M, N, num_iters, false, sm_count);
+    if (N <= 128 || g_swap_two_sm == 0 || g_path_mode == 6) return one;
+    const SwapPlan two = plan_swap(M, N, num_iters, true, sm_count);
+    if (g_swap_two_sm == 1 || g_path_mode == 5 || !one.pw) return two;
+    return two.pw && two.cycles + SWAP_PAIR_FIXED_CYCLES < one.cycles ? two : one;
+}
+
 template <bool CONV, bool TWO_SM>
 static int launch_swap(DeviceCtx* ctx, int slot, const SwapPlan& pl, const CUtensorMap& tmW, const CUtensorMap& tmX, const SwapParams& p,
                        cudaStream_t st) {
@@ -683,22 +699,22 @@ static int run_swap(DeviceCtx* ctx, bool conv, const SwapPlan& pl, const CUtenso
 // Whether a problem goes to the channel-major kernel.  Forced (path mode 4, I8OPS_SWAP=2): whenever it is legal.  By
 // rule: its read-out costs more per output than the large-tile kernel's (a transpose in registers), so it is taken only
 // where its freely chosen strip width buys occupancy: the large-tile plan would leave at least a fifth more of the chip
-// idle than the channel-major plan (the 3x3 layers with 12544 pixels and 256 filters: 98 tiles on 148 SMs against 72
-// strips on 74 CTA pairs; measured 8.6 -> 8.0 us and 11.4 -> 9.9 us), on problems with enough K per tile for that to
+// idle than the channel-major plan (the 3x3 layers with 12544 pixels and 256 filters: 98 tiles on 148 SMs against 144
+// strips of 128 channels x 176 pixels; measured 8.6 -> 7.7 us and 11.4 -> 9.6 us), on problems with enough K per tile for that to
 // matter and too small for the 256 x 256 pair kernel.
 static bool swap_wanted(bool conv, int M, int N, int K, int num_kb, int num_iters, int num_kblocks, int cb, int sm_count) {
-    if (g_path_mode == 4 || g_swap == 2) return true;
+    if (g_path_mode >= 4 || g_swap == 2) return true;
     if (!g_swap || g_path_mode != 0 || g_force_bn >= 0) return false;
     if (N < 256 || num_iters < 8) return false;
     if (!conv && recorded_plan(M, N, K)) return false;      // a schedule recorded for this shape's class takes precedence
     const TcPlan old_plan = plan_tc(conv, M, N, K, num_kb, num_iters, num_kblocks, cb, sm_count);
     if (old_plan.two_sm || 2 * old_plan.num_tiles < sm_count) return false;   // tiny problems: launch latency, not occupancy, bounds them
-    const SwapPlan sp = plan_swap(M, N, num_iters, true, sm_count);
+    const SwapPlan sp = plan_swap_auto(M, N, num_iters, sm_count);
     if (!sp.pw) return false;
     const int waves_old = (old_plan.num_tiles + sm_count - 1) / sm_count;
     const double eff_old = (double)old_plan.num_tiles / ((double)waves_old * sm_count);
-    const int pairs = sm_count / 2, waves_new = (sp.num_tiles + pairs - 1) / pairs;
-    const double eff_new = (double)sp.num_tiles / ((double)waves_new * pairs);
+    const int workers = sp.two_sm ? sm_count / 2 : sm_count, waves_new = (sp.num_tiles + workers - 1) / workers;
+    const double eff_new = (double)sp.num_tiles / ((double)waves_new * workers);
     return eff_new - eff_old >= 0.2;
 }
 
@@ -706,7 +722,7 @@ static int run_gemm_swap(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int
                          const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N, int K,
                          int relu, cudaStream_t st, const float* fscale) {
     const KLoop kl = gemm_kloop(K);
-    const SwapPlan pl = plan_swap(M, N, kl.num_iters, N > 128, ctx->sm_count);
+    const SwapPlan pl = plan_swap_auto(M, N, kl.num_iters, ctx->sm_count);
     if (!pl.pw || pl.stages < 2) return I8_ERR_UNSUPPORTED;
     CUtensorMap tmX;
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
@@ -735,7 +751,7 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     t_used_swap = false;
     if (swap_wanted(true, M, Kf, K, (K + BK - 1) / BK, kl.num_iters, kl.num_kblocks, cb, ctx->sm_count)) {
         // filters on the tensor-memory lanes, a strip of output pixels on the columns
-        const SwapPlan sp = plan_swap(M, Kf, kl.num_iters, Kf > 128, ctx->sm_count);
+        const SwapPlan sp = plan_swap_auto(M, Kf, kl.num_iters, ctx->sm_count);
         if (sp.pw && sp.stages >= 2) {
             CUtensorMap tmX;
             int rc = make_tmap_im2col(&tmX, x, N, H, W, C, R, S, stride_h, stride_w, pad_h, pad_w, cb, sp.b_rows, swizzle_for(cb));
@@ -1346,7 +1362,7 @@ int i8ops_plan_gemm(int M, int N, int K, int sm_count, i8_plan* out) {
     if (M <= 0 || N <= 0 || K <= 0 || sm_count <= 0) return I8_ERR_SHAPE;
     const KLoop kl = gemm_kloop(K);
     if (swap_wanted(false, M, N, K, kl.num_kblocks, kl.num_iters, kl.num_kblocks, BK, sm_count)) {
-        const SwapPlan sp = plan_swap(M, N, kl.num_iters, N > 128, sm_count);
+        const SwapPlan sp = plan_swap_auto(M, N, kl.num_iters, sm_count);
         if (sp.pw && sp.stages >= 2) { fill_plan_swap(sp, M, N, out); return I8_OK; }
     }
     fill_plan(plan_tc(false, M, N, K, kl.num_kblocks, kl.num_iters, kl.num_kblocks, BK, sm_count), out);
@@ -1407,7 +1423,7 @@ int i8ops_last_path(void) { return t_last_path; }
 
 int i8ops_set_path(int mode) {
     const int prev = g_path_mode;
-    if (mode >= 0 && mode <= 4) g_path_mode = mode;
+    if (mode >= 0 && mode <= 6) g_path_mode = mode;
     return prev;
 }
 

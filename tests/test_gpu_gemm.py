@@ -333,8 +333,9 @@ def test_recorded_class_plan_runs_and_is_reported():
     p = inputs.make_gemm(12544, 256, 1152, 4150, per_channel=1, relu=1)
     got = H.gemm_gpu(p)
     ran, asked = i8.last_plan(), i8.plan_gemm(p.M, p.N, p.K)
-    assert i8.last_path() == i8.PATH_CHANNEL_MAJOR_2SM and ran["kernel"] == 1 and ran == asked
-    assert ran["tile_n"] == 256 and ran["tile_m"] % 16 == 0 and ran["m_tiles"] * ran["tile_m"] >= p.M and ran["workers"] <= 74
+    assert i8.last_path() == i8.PATH_CHANNEL_MAJOR and ran["kernel"] == 1 and ran == asked
+    assert ran["tile_n"] == 128 and ran["cta_group"] == 1 and ran["tile_m"] % 16 == 0
+    assert ran["m_tiles"] * ran["tile_m"] >= p.M and ran["n_tiles"] == 2 and ran["workers"] <= 148
     H.assert_same(got, H.gemm_oracle(p), p.name)
     # without a recorded entry nearby, what ran is still what the query reports (config 1a: CTA pairs by the rule)
     p = inputs.make_gemm(2048, 2304, 1024, 4200, per_channel=1, relu=0)

@@ -36,10 +36,15 @@ def test_gemm_shapes(M, N, K):
         p = inputs.make_gemm(M, N, K, 6000 + M + N + K, per_channel=per_channel, relu=relu, shift_lo=12, shift_hi=22,
                              lda_pad=pad, ldb_pad=pad, ldc_pad=16 * per_channel)
         want = H.gemm_oracle(p)
-        i8.set_path(4)
-        got = H.gemm_gpu(p)
-        assert i8.last_path() == (i8.PATH_CHANNEL_MAJOR_2SM if N > 128 else i8.PATH_CHANNEL_MAJOR), i8.last_path()
-        H.assert_same(got, want, p.name)
+        # 4: single CTAs or CTA pairs by the cost model; 5: pairs whenever there are more than 128 channels; 6: single CTAs
+        for mode in (4, 5, 6):
+            i8.set_path(mode)
+            got = H.gemm_gpu(p)
+            if mode == 4:
+                assert i8.last_path() in _swap_paths(), i8.last_path()
+            else:
+                assert i8.last_path() == (i8.PATH_CHANNEL_MAJOR_2SM if N > 128 and mode == 5 else i8.PATH_CHANNEL_MAJOR), i8.last_path()
+            H.assert_same(got, want, f"{p.name} mode {mode}")
     assert i8.last_device_status() == 0
 
 
@@ -103,11 +108,11 @@ def test_conv_shapes(shape):
     N, Hh, W, C, K, R, S, st, pad = shape
     p = inputs.make_conv(N, Hh, W, C, K, R, S, st, pad, 6200 + sum(shape))
     want = H.conv_oracle(p)
-    i8.set_path(4)
-    got = H.conv_gpu(p)
-    if R == 1 and S == 1 or p.x.size >= 131072:
-        assert i8.last_path() in _swap_paths(), i8.last_path()
-    H.assert_same(got, want, p.name)
+    for mode in (4, 5, 6):
+        i8.set_path(mode)
+        got = H.conv_gpu(p)
+        assert i8.last_path() in _swap_paths(), i8.last_path()      # small activation tensors: unfold pass + this kernel
+        H.assert_same(got, want, f"{p.name} mode {mode}")
     assert i8.last_device_status() == 0
 
 
@@ -117,10 +122,11 @@ def test_config3_conv_mix_channel_major(j):
     import paper_2505_18574_b200 as i8
     p = inputs.config3(j)
     want = H.conv_oracle(p)
-    i8.set_path(4)
-    got = H.conv_gpu(p)
-    assert i8.last_path() == i8.PATH_CHANNEL_MAJOR_2SM
-    H.assert_same(got, want, p.name)
+    for mode in (5, 6):
+        i8.set_path(mode)
+        got = H.conv_gpu(p)
+        assert i8.last_path() == (i8.PATH_CHANNEL_MAJOR_2SM if mode == 5 else i8.PATH_CHANNEL_MAJOR)
+        H.assert_same(got, want, f"{p.name} mode {mode}")
     H.not_degenerate(want)
 
 
@@ -141,12 +147,15 @@ def test_float_scale_readout(M, N, K, per_channel, relu):
     want = oracle.gemm_i8_fscale(p.A, p.a_rs, 1, p.B, 1, p.b_cs, N, p.bias, scale, per_channel, M, N, K, relu)
     A = torch.from_numpy(p.A).cuda()[:, :K]; B = torch.from_numpy(p.B).cuda()[:, :K]
     bias = torch.from_numpy(p.bias).cuda(); sc = torch.from_numpy(scale).cuda()
-    for mode in (0, 1):
+    for mode in (0, 1, 5, 6):
         i8.set_path(mode)
         C = torch.full((M, N), 0x5A, dtype=torch.int8, device="cuda")
         i8.gemm_i8_fscale(A, B.t(), C, bias, sc, per_channel, relu)
         assert i8.last_device_status() == 0
-        assert i8.last_path() == (i8.PATH_GENERIC if mode == 1 else (i8.PATH_CHANNEL_MAJOR_2SM if N > 128 else i8.PATH_CHANNEL_MAJOR))
+        if mode == 0:
+            assert i8.last_path() in _swap_paths()
+        else:
+            assert i8.last_path() == (i8.PATH_GENERIC if mode == 1 else (i8.PATH_CHANNEL_MAJOR_2SM if N > 128 and mode == 5 else i8.PATH_CHANNEL_MAJOR))
         H.assert_same(C.cpu().numpy(), want, f"float scale mode {mode}")
     H.not_degenerate(want)
     # large accumulators: |t| above 2^24 is rounded by the conversion itself
