@@ -77,9 +77,23 @@ __device__ __forceinline__ SwapChan make_swap_chan(int32_t bias, int32_t mult, i
 }
 
 // Requantise `count` (16 or 32) accumulators of one channel and pack them four to a word.
+// `all_fold`: every lane of the warp is in the folded form (the common case: positive scales below one half), known
+// warp-uniformly, so that the hot path is straight-line code without a per-lane branch.
 template <int COUNT>
-__device__ __forceinline__ void swap_requant(const int32_t (&v)[32], const SwapChan& ch, int relu, uint32_t (&out)[8]) {
-    if (ch.form == 0) {
+__device__ __forceinline__ void swap_requant(const int32_t (&v)[32], const SwapChan& ch, int relu, bool all_fold, uint32_t (&out)[8]) {
+    if (all_fold) {
+        if (relu) {
+#pragma unroll
+            for (int j = 0; j < COUNT / 4; j++)
+                out[j] = relu_s8x4(pack_sat4(requant_fold(v[4 * j + 0], ch.m2, ch.c64), requant_fold(v[4 * j + 1], ch.m2, ch.c64),
+                                             requant_fold(v[4 * j + 2], ch.m2, ch.c64), requant_fold(v[4 * j + 3], ch.m2, ch.c64)));
+        } else {
+#pragma unroll
+            for (int j = 0; j < COUNT / 4; j++)
+                out[j] = pack_sat4(requant_fold(v[4 * j + 0], ch.m2, ch.c64), requant_fold(v[4 * j + 1], ch.m2, ch.c64),
+                                   requant_fold(v[4 * j + 2], ch.m2, ch.c64), requant_fold(v[4 * j + 3], ch.m2, ch.c64));
+        }
+    } else if (ch.form == 0) {
 #pragma unroll
         for (int j = 0; j < COUNT / 4; j++) {
             const uint32_t pk = pack_sat4(requant_fold(v[4 * j + 0], ch.m2, ch.c64), requant_fold(v[4 * j + 1], ch.m2, ch.c64),
@@ -350,6 +364,7 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         uint32_t acc_phase = 0;
         bool dead = false;
         SwapChan ch = make_swap_chan(0, 0, 0, 0);
+        bool all_fold = false;
         int n = 0;
         for (int tile = first_tile; tile < p.num_tiles; tile += tile_step) {
             const int m_tile = fast_div(tile, p.n_blocks, p.inv_nb), n_blk = tile - m_tile * p.n_blocks;
@@ -365,6 +380,7 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                 }
                 ch = make_swap_chan(bias, mult, shift, p.relu);
                 if (p.fscale) { ch.form = 3; ch.fscale = fs; }
+                all_fold = __all_sync(0xffffffffu, ch.form == 0);
                 cached_n_blk = n_blk;
             }
             if (!dead) dead = !__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * ab, acc_phase, env, DEV_TIMEOUT_EPILOGUE));
@@ -383,11 +399,11 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                 if (width == 32) {
                     tmem_ld_32x32(t0 + col, v);
                     tmem_ld_wait();
-                    swap_requant<32>(v, ch, p.relu, out);
+                    swap_requant<32>(v, ch, p.relu, all_fold, out);
                 } else {
                     tmem_ld_32x16(t0 + col, v);
                     tmem_ld_wait();
-                    swap_requant<16>(v, ch, p.relu, out);
+                    swap_requant<16>(v, ch, p.relu, all_fold, out);
                 }
                 if (p.c_word_ok) {
                     // word j: channels n_quad .. n_quad + 3 of output row m0 + col + 4j + pix
