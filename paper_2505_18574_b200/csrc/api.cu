@@ -629,7 +629,6 @@ static SwapPlan plan_swap(int M, int N, int num_iters, bool two_sm, int sm_count
     int stages = (226 * 1024 - fixed) / stage_bytes;
     if (stages > SWAP_MAX_STAGES) stages = SWAP_MAX_STAGES;
     if (g_swap_stages >= 2 && g_swap_stages < stages) stages = g_swap_stages;
-    stages &= ~1;                                        // two producers alternate ring slots
     best.stages = stages;
     best.off_b = stages * 16384;
     best.off_bar = best.off_b + stages * b_stage;

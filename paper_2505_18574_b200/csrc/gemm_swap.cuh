@@ -232,7 +232,7 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         // ------------------------------------------------------------------ producer (whole warp loops, one lane issues)
         const int pid = warp == 0 ? 0 : 1;
         int stage = 0;
-        uint32_t phase = 0, issued = 0, issued_phase = 0;
+        uint32_t phase = 0, issued = 0, issued_phase = 0, seq = 0;     // seq: ring slots filled so far by both producers together
         bool ok = true, first_pass = true;
         const bool leader = elect_one();
         const uint32_t stage_tx = a_sub_bytes + b_sub_bytes;
@@ -252,9 +252,12 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             int c_idx = 0, fs = 0, fr = 0;
             for (int kbi = 0; kbi < kl.num_kblocks;) {
                 const int nb = min(kl.nsub, kl.num_kblocks - kbi);
-                if (NPROD == 2 && (stage & 1) != pid) {
+                if (NPROD == 2 && (seq & 1) != (uint32_t)pid) {
+                    // the other producer's turn (turns alternate along the sequence of slots, so the ring may have an odd
+                    // number of them): only keep the counters in step
                     for (int j = 0; j < nb; j++, kbi++)
                         if (CONV && ++c_idx == kl.cblocks) { c_idx = 0; if (++fs == kl.S) { fs = 0; ++fr; } }
+                    ++seq;
                     if (++stage == stages) { stage = 0; phase ^= 1; first_pass = false; }
                     continue;
                 }
@@ -281,6 +284,7 @@ gemm_i8_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                 }
                 issued |= 1u << stage;
                 issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
+                ++seq;
                 if (++stage == stages) { stage = 0; phase ^= 1; first_pass = false; }
             }
         }
