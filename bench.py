@@ -357,6 +357,7 @@ def main():
         from paper_2505_18574_b200 import bench_details
         pk = measured_peaks()
         if not args.no_details:
+            time.sleep(0.5)             # the per-configuration timings start from an idle GPU, not from the power-capped clock
             details = bench_details.run(dev, peak_tops=2 * pk["bf16_burst"], peak_gbs=pk["hbm_gbs"], oracle=oracle_t)
         # this library's own tensor-core issue-rate probe (operands resident in shared memory): burst and sustained
         probe = bench_details.run_peak(dev)
