@@ -79,8 +79,12 @@ typedef enum {
  *   C      device, int8, row-major, ldc >= N.
  *   bias   device, int32[N], or NULL.
  *   mult, shift, per_channel, relu   see the epilogue above.
- * The tensor path needs both operands K-contiguous (a_cs == 1, b_rs == 1) with 16-byte aligned base
- * addresses and leading dimensions; anything else is computed by the generic kernel, same results.
+ * The tensor path fetches operands in place when their base addresses and leading dimensions are multiples of 16 bytes
+ * (either storage order of either operand).  Other operands are first packed into K-contiguous, zero-padded copies in a
+ * workspace that is allocated and released in stream order from a memory pool the library keeps per device (the call
+ * stays asynchronous and may be captured into a CUDA graph; make the first such call on a device outside any capture);
+ * problems below 2^18 multiply-accumulates, or whose copies would exceed 256 MiB, take the one-thread-per-output kernel
+ * instead.  Same results on every path.  i8ops_last_gemm_packed() tells whether the last call packed its operands.
  * Errors: I8_ERR_NULL, I8_ERR_SHAPE (negative M, N or K), I8_ERR_STRIDE, I8_ERR_RANGE, I8_ERR_CUDA.
  * M == 0 or N == 0 returns I8_OK and launches nothing; K == 0 yields epilogue(0).
  */
@@ -142,9 +146,11 @@ int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs,
  *   y  device int8 [N][P][Q][K] (dense),  P = floor((H + 2*pad_h - R)/stride_h) + 1, Q likewise.
  *   bias/mult/shift indexed by filter k.
  * Layers that the implicit-GEMM loads do not take (an activation tensor below 128 KiB, a stride above 8, a filter side or
- * padding above 16) run, when C % 16 == 0, as an unfold pass into the GEMM form's A matrix followed by the tensor GEMM;
- * that matrix (N*P*Q x R*S*C bytes, at most 256 MiB) is allocated and released in stream order from a memory pool the
- * library keeps per device, so the call stays asynchronous and may be captured into a CUDA graph.
+ * padding above 16, a channel count that is not a multiple of 32, misaligned bases) run as an unfold pass into the GEMM
+ * form's A matrix followed by the tensor GEMM; that matrix (N*P*Q rows of R*S*C bytes rounded up to 16, plus a padded
+ * copy of the filters when C % 16 != 0; at most 256 MiB together, else the one-thread-per-output kernel serves the call)
+ * is allocated and released in stream order from a memory pool the library keeps per device, so the call stays
+ * asynchronous and may be captured into a CUDA graph.
  * The first such call on a device creates the pool: make it outside any stream capture.
  * i8ops_last_conv_unfolded() tells whether the most recent convolution of this thread ran that way.
  * Errors: I8_ERR_NULL, I8_ERR_SHAPE (a non-positive extent or an empty output), I8_ERR_UNSUPPORTED
@@ -156,6 +162,8 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y,
               int stride_h, int stride_w, int pad_h, int pad_w, int relu, void* stream);
 
 int i8ops_last_conv_unfolded(void);
+/* Whether the most recent gemm_i8 of this thread ran on packed copies of its operands (see gemm_i8). */
+int i8ops_last_gemm_packed(void);
 
 /*
  * Host-buffer variants: every pointer is HOST memory (pinned memory makes the copies asynchronous).

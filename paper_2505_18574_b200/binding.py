@@ -44,6 +44,7 @@ SIGNATURES = {
     "i8ops_last_cuda_error": (_int, []),
     "i8ops_last_path": (_int, []),
     "i8ops_last_conv_unfolded": (_int, []),
+    "i8ops_last_gemm_packed": (_int, []),
     "i8ops_set_path": (_int, [_int]),
     "i8ops_set_wait_limit_ms": (None, [_int]),
     "i8ops_version": (_int, []),
@@ -268,6 +269,11 @@ def set_class_plan(shape_class: int, base=(0, 0, 0), tile_n: int = 0, cta_group:
 def last_conv_unfolded() -> bool:
     """Whether the calling thread's most recent convolution ran as an unfold pass followed by the tensor GEMM."""
     return bool(lib().i8ops_last_conv_unfolded())
+
+
+def last_gemm_packed() -> bool:
+    """Whether the calling thread's most recent gemm_i8 ran on packed copies of operands the tensor path could not fetch in place."""
+    return bool(lib().i8ops_last_gemm_packed())
 
 
 def tmap_cache_stats():

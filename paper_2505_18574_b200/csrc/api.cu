@@ -63,6 +63,7 @@ static thread_local int t_last_path = I8_PATH_NONE;
 static thread_local int t_last_cuda = 0;
 static thread_local bool t_used_two_sm = false;
 static thread_local bool t_used_swap = false;     // the last tensor-path launch was the channel-major kernel
+static thread_local bool t_last_packed = false;   // the last GEMM ran on packed copies of its operands
 static thread_local bool t_last_unfold = false;   // the last convolution ran as unfold + tensor GEMM
 static thread_local bool t_tmap_failed = false;   // the last tensor-path attempt stopped at a tensor-map encoding (nothing launched)
 
@@ -769,17 +770,12 @@ static int run_conv_tc(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t*
     return run_tc(ctx, true, pl, tmA, kl, w, K, y, Kf, bias, mult, shift, per_channel, M, Kf, K, relu, st);
 }
 
-// Convolutions the im2col tensor maps do not take (small activation tensors, long strides, large filters) with
-// C % 16 == 0: the activations are unfolded into the GEMM form's A matrix in a workspace that lives in stream order
-// (allocated from the library's own pool before the two launches and released behind them, so concurrent streams never
-// share it and a captured graph owns its copy), then the product runs on the tensor path.  Returns I8_ERR_UNSUPPORTED,
-// launching nothing, when the workspace would be too large or cannot be had.
-static const int64_t UNFOLD_MAX_BYTES = 256ll << 20;
-static int run_conv_unfold(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, const int32_t* mult,
-                           const int32_t* shift, int per_channel, int N, int H, int W, int C, int Kf, int R, int S, int P, int Q,
-                           int stride_h, int stride_w, int pad_h, int pad_w, int relu, cudaStream_t st) {
-    const int64_t M = (int64_t)N * P * Q, K = (int64_t)R * S * C;
-    if (C % 16 != 0 || M >= (1ll << 31) || M * K > UNFOLD_MAX_BYTES) return I8_ERR_UNSUPPORTED;
+// Stream-ordered workspaces: a memory pool the library creates per device on first use.  A block is allocated on the
+// caller's stream before the launches that use it and released behind them (release threshold unlimited, so the next call
+// reuses it): concurrent streams never share a block, the calls stay asynchronous, and a captured graph owns its copy.
+static const int64_t WORKSPACE_MAX_BYTES = 256ll << 20;
+static int pool_alloc(DeviceCtx* ctx, void** out, int64_t bytes, cudaStream_t st) {
+    if (bytes <= 0 || bytes > WORKSPACE_MAX_BYTES) return I8_ERR_UNSUPPORTED;
     if (!ctx->pool_ready.load(std::memory_order_acquire)) {
         std::lock_guard<std::mutex> lock(g_mutex);
         if (!ctx->pool_ready.load(std::memory_order_relaxed)) {
@@ -791,25 +787,97 @@ static int run_conv_unfold(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int
             props.location.type = cudaMemLocationTypeDevice;
             props.location.id = dev;
             if (cudaMemPoolCreate(&ctx->pool, &props) != cudaSuccess) { cudaGetLastError(); return I8_ERR_UNSUPPORTED; }
-            uint64_t keep = ~0ull;                  // released blocks stay in the pool: the next call reuses them
+            uint64_t keep = ~0ull;
             cudaMemPoolSetAttribute(ctx->pool, cudaMemPoolAttrReleaseThreshold, &keep);
             ctx->pool_ready.store(true, std::memory_order_release);
         }
     }
-    void* a = nullptr;
-    if (cudaMallocFromPoolAsync(&a, (size_t)(M * K), ctx->pool, st) != cudaSuccess) { cudaGetLastError(); return I8_ERR_UNSUPPORTED; }
-    UnfoldParams u{x, (int8_t*)a, N, H, W, C, R, S, P, Q, stride_h, stride_w, pad_h, pad_w};
-    const int64_t pieces = M * K / 16;
-    int64_t blocks = (pieces + 255) / 256;
+    if (cudaMallocFromPoolAsync(out, (size_t)bytes, ctx->pool, st) != cudaSuccess) { cudaGetLastError(); return I8_ERR_UNSUPPORTED; }
+    return I8_OK;
+}
+
+static int grid_for(int64_t items) {
+    int64_t blocks = (items + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    conv_unfold_i8_kernel<<<(int)blocks, 256, 0, st>>>(u);
+    return (int)(blocks < 1 ? 1 : blocks);
+}
+
+static int launch_pack(const int8_t* src, int64_t rs, int64_t cs, int rows, int K, int kp, int8_t* dst, cudaStream_t st) {
+    PackParams pk{src, dst, rs, cs, rows, K, kp};
+    pack_rows_i8_kernel<<<grid_for((int64_t)rows * (kp / 16)), 256, 0, st>>>(pk);
     const cudaError_t le = cudaGetLastError();
-    int rc = le == cudaSuccess ? I8_OK : cuda_fail(le);
+    return le == cudaSuccess ? I8_OK : cuda_fail(le);
+}
+
+static int64_t up256(int64_t v) { return (v + 255) & ~(int64_t)255; }
+
+// Convolutions the im2col tensor maps do not take (small activation tensors, long strides, large filters, channel counts
+// that are not a multiple of 32): the activations are unfolded into the GEMM form's A matrix in a stream-ordered
+// workspace, then the product runs on the tensor path.  With C % 16 != 0 the rows of that matrix and of a repacked copy
+// of the filters are padded with zeros to a multiple of 16 bytes.  Returns I8_ERR_UNSUPPORTED, launching nothing, when
+// the workspace would be too large or cannot be had.
+static int run_conv_unfold(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, const int32_t* mult,
+                           const int32_t* shift, int per_channel, int N, int H, int W, int C, int Kf, int R, int S, int P, int Q,
+                           int stride_h, int stride_w, int pad_h, int pad_w, int relu, cudaStream_t st) {
+    const int64_t M = (int64_t)N * P * Q, K = (int64_t)R * S * C;
+    if (M >= (1ll << 31)) return I8_ERR_UNSUPPORTED;
+    const bool whole_pieces = C % 16 == 0 && aligned16(x) && aligned16(w);
+    const int64_t kp = (K + 15) & ~(int64_t)15;
+    const int64_t a_bytes = up256(M * kp), w_bytes = whole_pieces ? 0 : up256((int64_t)Kf * kp);
+    void* ws = nullptr;
+    int rc = pool_alloc(ctx, &ws, a_bytes + w_bytes, st);
+    if (rc) return rc;
+    int8_t* a = (int8_t*)ws;
+    const int8_t* wmat = w;
+    cudaError_t le;
+    if (whole_pieces) {
+        UnfoldParams u{x, a, N, H, W, C, R, S, P, Q, stride_h, stride_w, pad_h, pad_w};
+        conv_unfold_i8_kernel<<<grid_for(M * K / 16), 256, 0, st>>>(u);
+        le = cudaGetLastError();
+    } else {
+        UnfoldBytesParams u{x, a, N, H, W, C, R, S, P, Q, stride_h, stride_w, pad_h, pad_w, (int)kp};
+        conv_unfold_bytes_i8_kernel<<<grid_for(M * (kp / 16)), 256, 0, st>>>(u);
+        le = cudaGetLastError();
+        if (le == cudaSuccess) {
+            rc = launch_pack(w, K, 1, Kf, (int)K, (int)kp, a + a_bytes, st);
+            wmat = a + a_bytes;
+        }
+    }
+    if (le != cudaSuccess) rc = cuda_fail(le);
     if (rc == I8_OK) {
         t_used_two_sm = false; t_tmap_failed = false;
-        rc = run_gemm_tc(ctx, (const int8_t*)a, K, w, K, y, Kf, bias, mult, shift, per_channel, (int)M, Kf, (int)K, relu, st);
+        rc = run_gemm_tc(ctx, a, kp, wmat, kp, y, Kf, bias, mult, shift, per_channel, (int)M, Kf, (int)kp, relu, st);
     }
-    cudaFreeAsync(a, st);
+    cudaFreeAsync(ws, st);
+    return rc;
+}
+
+// GEMM operands the tensor path cannot fetch in place (a base or leading dimension that is not a multiple of 16 bytes,
+// general strides): packed into K-contiguous, zero-padded copies in a stream-ordered workspace, then the tensor path.
+// Operands that are already in a legal layout are used where they are.
+static int run_gemm_packed(DeviceCtx* ctx, const int8_t* A, int64_t a_rs, int64_t a_cs, bool a_ok, const int8_t* B, int64_t b_rs,
+                           int64_t b_cs, bool b_ok, int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult,
+                           const int32_t* shift, int per_channel, int M, int N, int K, int relu, cudaStream_t st) {
+    const int64_t kp = ((int64_t)K + 15) & ~(int64_t)15;
+    const int64_t a_bytes = a_ok ? 0 : up256((int64_t)M * kp), b_bytes = b_ok ? 0 : up256((int64_t)N * kp);
+    void* ws = nullptr;
+    int rc = pool_alloc(ctx, &ws, a_bytes + b_bytes, st);
+    if (rc) return rc;
+    const int8_t* Ap = A; int64_t lda = a_rs;
+    const int8_t* Bp = B; int64_t ldb = b_cs;
+    if (!a_ok) {
+        rc = launch_pack(A, a_rs, a_cs, M, K, (int)kp, (int8_t*)ws, st);
+        Ap = (int8_t*)ws; lda = kp;
+    }
+    if (rc == I8_OK && !b_ok) {
+        rc = launch_pack(B, b_cs, b_rs, N, K, (int)kp, (int8_t*)ws + a_bytes, st);      // row n of the copy = column n of B
+        Bp = (int8_t*)ws + a_bytes; ldb = kp;
+    }
+    if (rc == I8_OK) {
+        t_used_two_sm = false; t_tmap_failed = false;
+        rc = run_gemm_tc(ctx, Ap, lda, Bp, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
+    }
+    cudaFreeAsync(ws, st);
     return rc;
 }
 
@@ -959,6 +1027,7 @@ int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_
             const int32_t* bias, const int32_t* mult, const int32_t* shift, int per_channel, int M, int N, int K, int relu,
             void* stream) {
     t_last_path = I8_PATH_NONE;
+    t_last_packed = false;
     int rc = validate_gemm(A, a_rs, a_cs, B, b_rs, b_cs, C, ldc, mult, shift, M, N, K);
     if (rc) return rc;
     if (M == 0 || N == 0) return I8_OK;
@@ -977,6 +1046,13 @@ int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_
         if (rc == I8_OK) t_last_path = tensor_path_used();
         if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         // the driver refused a tensor map for this geometry: nothing was launched, the generic kernel serves it
+    } else if (g_path_mode != 1 && g_unfold && K >= 1 && (int64_t)M * N * K >= (1ll << 18)) {
+        // operands the tensor path cannot fetch in place: packed copies in a stream-ordered workspace (tiny problems are
+        // quicker on the generic kernel than behind two extra launches)
+        rc = run_gemm_packed(ctx, A, a_rs, a_cs, a_k && aligned16(A), B, b_rs, b_cs, b_k && aligned16(B), C, ldc, bias, mult, shift,
+                             per_channel, M, N, K, relu, st);
+        if (rc == I8_OK) { t_last_path = tensor_path_used(); t_last_packed = true; return rc; }
+        if (rc != I8_ERR_UNSUPPORTED && !(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
     }
     GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, C, ldc, 0, bias, 0, mult, shift, per_channel, relu, 1, M, N, K, nullptr, 0, 0, 0};
     rc = run_gemm_generic(g, st);
@@ -1141,7 +1217,7 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
             if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
     }
-    if (g_path_mode != 1 && g_unfold && aligned16(x) && aligned16(w)) {
+    if (g_path_mode != 1 && g_unfold) {
         rc = run_conv_unfold(ctx, x, w, y, bias, mult, shift, per_channel, N, H, W, C, K, R, S, P, Q, stride_h, stride_w,
                              pad_h, pad_w, relu, st);
         if (rc == I8_OK) { t_last_path = tensor_path_used(); t_last_unfold = true; return rc; }
@@ -1158,6 +1234,7 @@ int conv2d_i8(const int8_t* x, const int8_t* w, int8_t* y, const int32_t* bias, 
 }
 
 int i8ops_last_conv_unfolded(void) { return t_last_unfold ? 1 : 0; }
+int i8ops_last_gemm_packed(void) { return t_last_packed ? 1 : 0; }
 
 int gemm_i8_host(const int8_t* A, const int8_t* B, int8_t* C, const int32_t* bias, const int32_t* mult, const int32_t* shift,
                  int per_channel, int M, int N, int K, int relu, void* stream) {

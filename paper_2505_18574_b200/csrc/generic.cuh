@@ -105,6 +105,66 @@ __global__ void __launch_bounds__(256) conv_unfold_i8_kernel(const UnfoldParams 
     }
 }
 
+// The same for any channel count: the matrix rows are padded with zeros to `kp` (a multiple of 16) bytes, one 16-byte
+// piece per thread and step, every byte placed on its own.
+struct UnfoldBytesParams {
+    const int8_t* x; int8_t* a;
+    int N, H, W, C, R, S, P, Q, stride_h, stride_w, pad_h, pad_w;
+    int kp;
+};
+
+__global__ void __launch_bounds__(256) conv_unfold_bytes_i8_kernel(const UnfoldBytesParams p) {
+    const int per_row = p.kp >> 4, K = p.R * p.S * p.C;
+    const int64_t total = (int64_t)p.N * p.P * p.Q * per_row;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int piece = (int)(idx % per_row);
+        int64_t rest = idx / per_row;
+        const int q = (int)(rest % p.Q); rest /= p.Q;
+        const int pp = (int)(rest % p.P);
+        const int n = (int)(rest / p.P);
+        uint32_t w4[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+            const int k = piece * 16 + j;
+            int8_t v = 0;
+            if (k < K) {
+                const int c = k % p.C, rs = k / p.C, s = rs % p.S, r = rs / p.S;
+                const int h = pp * p.stride_h - p.pad_h + r, ww = q * p.stride_w - p.pad_w + s;
+                if (h >= 0 && h < p.H && ww >= 0 && ww < p.W) v = p.x[(((int64_t)n * p.H + h) * p.W + ww) * p.C + c];
+            }
+            w4[j >> 2] |= (uint32_t)(uint8_t)v << (8 * (j & 3));
+        }
+        reinterpret_cast<int4*>(p.a)[idx] = make_int4((int)w4[0], (int)w4[1], (int)w4[2], (int)w4[3]);
+    }
+}
+
+// Copies a strided int8 matrix (element (r, k) at src[r * rs + k * cs]) into a K-contiguous one with rows of `kp` bytes
+// (a multiple of 16, zero-padded beyond K): the layout the tensor path wants, for operands whose bases or leading
+// dimensions are not multiples of 16 bytes or whose strides are general.
+struct PackParams {
+    const int8_t* src; int8_t* dst;
+    int64_t rs, cs;
+    int rows, K, kp;
+};
+
+__global__ void __launch_bounds__(256) pack_rows_i8_kernel(const PackParams p) {
+    const int per_row = p.kp >> 4;
+    const int64_t total = (int64_t)p.rows * per_row;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int piece = (int)(idx % per_row);
+        const int64_t r = idx / per_row;
+        const int8_t* row = p.src + r * p.rs;
+        uint32_t w4[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+            const int k = piece * 16 + j;
+            const int8_t v = k < p.K ? row[(int64_t)k * p.cs] : (int8_t)0;
+            w4[j >> 2] |= (uint32_t)(uint8_t)v << (8 * (j & 3));
+        }
+        reinterpret_cast<int4*>(p.dst)[idx] = make_int4((int)w4[0], (int)w4[1], (int)w4[2], (int)w4[3]);
+    }
+}
+
 // Self-test of the bounded wait: one CTA waits on an mbarrier that nothing ever signals.  The wait must give
 // up after `limit_cycles`, record DEV_TIMEOUT_TEST in the status word and return normally.
 __global__ void bounded_wait_selftest_kernel(long long limit_cycles, unsigned* dev_status) {

@@ -106,6 +106,25 @@ def test_conv_unfolded_layers_take_the_tensor_path(N, H_, W, C, K, R, S, st, pad
     assert not i8.last_conv_unfolded() and i8.last_path() == i8.PATH_GENERIC
 
 
+@pytest.mark.parametrize("N,H_,W,C,K,R,S,st,pad", [
+    (4, 32, 32, 3, 64, 7, 7, 2, 3),       # an RGB first layer: 147 columns padded to 160
+    (2, 15, 17, 20, 24, 3, 3, 1, 1),      # channels a multiple of 4 only
+    (3, 9, 9, 7, 5, 2, 2, 1, 0),          # odd everything
+    (16, 56, 56, 8, 32, 3, 3, 1, 1),      # a large activation tensor with 8 channels
+])
+def test_conv_with_any_channel_count_takes_the_tensor_path(N, H_, W, C, K, R, S, st, pad):
+    """Channel counts that are not a multiple of 16: byte-wise unfold, padded copy of the filters, tensor GEMM."""
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_conv(N, H_, W, C, K, R, S, st, pad, 1500 + N + H_ + C + K)
+    want = H.conv_oracle(p)
+    got = H.conv_gpu(p)
+    assert i8.last_conv_unfolded() and i8.last_path() in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM, i8.PATH_CHANNEL_MAJOR, i8.PATH_CHANNEL_MAJOR_2SM), i8.last_path()
+    H.assert_same(got, want, p.name + " unfolded byte-wise")
+    i8.set_path(1)
+    H.assert_same(H.conv_gpu(p), want, p.name + " generic")
+    assert not i8.last_conv_unfolded()
+
+
 def test_conv_unfolded_inside_a_cuda_graph_and_on_two_streams():
     """The unfold workspace lives in stream order: a captured graph owns its copy (replays give the same bytes), and two
     streams running different layers at once do not share it."""

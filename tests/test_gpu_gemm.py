@@ -37,6 +37,44 @@ def _both_paths(p, expect_tensor=True, two_sm=False):
     return want
 
 
+@pytest.mark.parametrize("M,N,K,lda_pad,ldb_pad,a_off,b_off", [
+    (200, 136, 100, 3, 5, 0, 0),         # leading dimensions that are not multiples of 16, ragged K
+    (512, 384, 256, 0, 0, 1, 0),         # A starts one byte off a 16-byte boundary, B is fetched in place
+    (300, 520, 272, 16, 0, 0, 7),        # B's base is off, A in place with a padded (still aligned) leading dimension
+    (1000, 96, 33, 1, 1, 3, 5),          # everything off at once
+    (4096, 1024, 512, 8, 8, 0, 0),       # large enough for 256-wide tiles
+])
+def test_operands_the_tensor_path_cannot_fetch_in_place_are_packed(M, N, K, lda_pad, ldb_pad, a_off, b_off):
+    """Misaligned bases and leading dimensions: packed copies in the stream-ordered workspace, then a tensor kernel."""
+    import torch
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_gemm(M, N, K, 4700 + M + N + K, per_channel=1, relu=M % 2, shift_lo=19, shift_hi=25, lda_pad=lda_pad, ldb_pad=ldb_pad)
+    want = H.gemm_oracle(p)
+    lda, ldb = p.A.shape[1], p.B.shape[1]
+
+    def shifted(host, off):
+        flat = torch.zeros(host.size + 16 + off, dtype=torch.int8, device="cuda")
+        base = (-flat.data_ptr()) % 16 + off                     # `off` bytes past a 16-byte boundary
+        flat[base:base + host.size] = torch.from_numpy(host.reshape(-1)).cuda()
+        return flat[base:base + host.size].view(host.shape)
+
+    A = shifted(p.A, a_off)[:, :K]; B = shifted(p.B, b_off)[:, :K]
+    assert A.data_ptr() % 16 == a_off and B.data_ptr() % 16 == b_off
+    bias, mult, shift = (torch.from_numpy(v).cuda() for v in (p.bias, p.mult, p.shift))
+    for mode in (0, 1):
+        i8.set_path(mode)
+        C = torch.full((M, N), 0x5A, dtype=torch.int8, device="cuda")
+        i8.gemm_i8(A, B.t(), C, bias, mult, shift, p.per_channel, p.relu)
+        assert i8.last_device_status() == 0
+        if mode == 0:
+            assert i8.last_gemm_packed() and i8.last_path() in TENSOR_PATHS, (i8.last_gemm_packed(), i8.last_path())
+        else:
+            assert not i8.last_gemm_packed() and i8.last_path() == i8.PATH_GENERIC
+        H.assert_same(C.cpu().numpy(), want, f"{p.name} mode {mode} lda {lda} ldb {ldb}")
+    i8.set_path(0)
+    H.not_degenerate(want)
+
+
 def test_config0_256cube():
     want = _both_paths(inputs.config0())
     H.not_degenerate(want)
