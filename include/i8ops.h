@@ -98,7 +98,8 @@ int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs,
  * Raw read-out: D[m*ldd + n] (+)= sum_k A[..] * B[..] as int32, with no bias, activation or scale.  This is the
  * accumulator read as accumulator-type data (Gemmini ISA description, continued: address bit 29 set), and with
  * accumulate != 0 the product is added to what D already holds (address bit 30: accumulate instead of overwrite),
- * which lets a caller split K across calls.  D is device int32, row-major, ldd >= N; other arguments as gemm_i8.
+ * which lets a caller split K across calls.  D is device int32, row-major, ldd >= N; other arguments as gemm_i8
+ * (misaligned operands are packed first, as there).
  * The sums must fit in int32 (always true for a single product with K <= 65536).
  * Errors: I8_ERR_NULL, I8_ERR_SHAPE, I8_ERR_STRIDE, I8_ERR_RANGE, I8_ERR_CUDA.
  */
@@ -114,8 +115,8 @@ int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs,
  * fl32 = rounding to IEEE-754 binary32 (nearest, ties to even), applied to the conversion of t and to the product;
  * rne = nearest integer, ties to even (the paper states no rounding rule; this is the reading taken).  A NaN product
  * yields 0.  scale: device, float[1] (per_channel == 0) or float[N].  Other arguments, layouts and errors as gemm_i8
- * (I8_ERR_NULL also for a NULL scale).  K-contiguous aligned operands run on the channel-major tensor kernel, anything
- * else on the generic kernel.
+ * (I8_ERR_NULL also for a NULL scale).  K-contiguous aligned operands run on the channel-major tensor kernel in place,
+ * other operands through packed copies as in gemm_i8.
  */
 int gemm_i8_fscale(const int8_t* A, int64_t a_rs, int64_t a_cs,
                    const int8_t* B, int64_t b_rs, int64_t b_cs,

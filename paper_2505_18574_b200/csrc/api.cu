@@ -857,7 +857,8 @@ static int run_conv_unfold(DeviceCtx* ctx, const int8_t* x, const int8_t* w, int
 // Operands that are already in a legal layout are used where they are.
 static int run_gemm_packed(DeviceCtx* ctx, const int8_t* A, int64_t a_rs, int64_t a_cs, bool a_ok, const int8_t* B, int64_t b_rs,
                            int64_t b_cs, bool b_ok, int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult,
-                           const int32_t* shift, int per_channel, int M, int N, int K, int relu, cudaStream_t st) {
+                           const int32_t* shift, int per_channel, int M, int N, int K, int relu, cudaStream_t st,
+                           const RawOut& raw = RawOut(), const float* fscale = nullptr) {
     const int64_t kp = ((int64_t)K + 15) & ~(int64_t)15;
     const int64_t a_bytes = a_ok ? 0 : up256((int64_t)M * kp), b_bytes = b_ok ? 0 : up256((int64_t)N * kp);
     void* ws = nullptr;
@@ -875,7 +876,12 @@ static int run_gemm_packed(DeviceCtx* ctx, const int8_t* A, int64_t a_rs, int64_
     }
     if (rc == I8_OK) {
         t_used_two_sm = false; t_tmap_failed = false;
-        rc = run_gemm_tc(ctx, Ap, lda, Bp, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st);
+        if (fscale) {
+            rc = run_gemm_swap(ctx, Ap, lda, Bp, ldb, C, ldc, bias, nullptr, nullptr, per_channel, M, N, K, relu, st, fscale);
+            if (rc == I8_OK) t_used_swap = true;
+        } else {
+            rc = run_gemm_tc(ctx, Ap, lda, Bp, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
+        }
     }
     cudaFreeAsync(ws, st);
     return rc;
@@ -1063,6 +1069,7 @@ int gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_
 int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_t b_rs, int64_t b_cs, int32_t* D, int64_t ldd,
                 int accumulate, int M, int N, int K, void* stream) {
     t_last_path = I8_PATH_NONE;
+    t_last_packed = false;
     if (M < 0 || N < 0 || K < 0) return I8_ERR_SHAPE;
     if (K > 65536) return I8_ERR_RANGE;
     if (M == 0 || N == 0) return I8_OK;
@@ -1083,6 +1090,12 @@ int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, in
                          a_m ? 1 : 0, b_n ? 1 : 0);
         if (rc == I8_OK) t_last_path = tensor_path_used();
         if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
+    } else if (g_path_mode != 1 && g_unfold && K >= 1 && (int64_t)M * N * K >= (1ll << 18)) {
+        RawOut raw; raw.D = D; raw.ldd = ldd; raw.accumulate = accumulate ? 1 : 0;
+        rc = run_gemm_packed(ctx, A, a_rs, a_cs, a_k && aligned16(A), B, b_rs, b_cs, b_k && aligned16(B), nullptr, 0, nullptr, nullptr,
+                             nullptr, 0, M, N, K, 0, st, raw);
+        if (rc == I8_OK) { t_last_path = tensor_path_used(); t_last_packed = true; return rc; }
+        if (rc != I8_ERR_UNSUPPORTED && !(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
     }
     GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, nullptr, 0, 0, nullptr, 0, nullptr, nullptr, 0, 0, 1, M, N, K,
                         D, ldd, 1, accumulate ? 1 : 0};
@@ -1094,6 +1107,7 @@ int gemm_i8_raw(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, in
 int gemm_i8_fscale(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B, int64_t b_rs, int64_t b_cs, int8_t* C, int64_t ldc,
                    const int32_t* bias, const float* scale, int per_channel, int M, int N, int K, int relu, void* stream) {
     t_last_path = I8_PATH_NONE;
+    t_last_packed = false;
     if (M < 0 || N < 0 || K < 0) return I8_ERR_SHAPE;
     if (K > 65536) return I8_ERR_RANGE;
     if (M == 0 || N == 0) return I8_OK;
@@ -1110,6 +1124,14 @@ int gemm_i8_fscale(const int8_t* A, int64_t a_rs, int64_t a_cs, const int8_t* B,
         t_used_two_sm = false; t_tmap_failed = false;
         rc = run_gemm_swap(ctx, A, a_rs, B, b_cs, C, ldc, bias, nullptr, nullptr, per_channel, M, N, K, relu, st, scale);
         if (rc == I8_OK) { t_used_swap = true; t_last_path = tensor_path_used(); return rc; }
+        if (rc != I8_ERR_UNSUPPORTED && !(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
+    } else if (g_path_mode != 1 && g_unfold && K >= 1 && (int64_t)M * N * K >= (1ll << 18)) {
+        // misaligned or M- / N-contiguous operands: packed K-contiguous copies, then the channel-major kernel
+        const bool a_ok = a_cs == 1 && a_rs % 16 == 0 && a_rs >= K && aligned16(A), b_ok = b_rs == 1 && b_cs % 16 == 0 && b_cs >= K && aligned16(B);
+        t_used_two_sm = false; t_tmap_failed = false;
+        rc = run_gemm_packed(ctx, A, a_rs, a_cs, a_ok, B, b_rs, b_cs, b_ok, C, ldc, bias, nullptr, nullptr, per_channel, M, N, K, relu, st,
+                             RawOut(), scale);
+        if (rc == I8_OK) { t_last_path = tensor_path_used(); t_last_packed = true; return rc; }
         if (rc != I8_ERR_UNSUPPORTED && !(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
     }
     GenericGemmParams g{A, a_rs, a_cs, 0, B, b_rs, b_cs, 0, C, ldc, 0, bias, 0, nullptr, nullptr, per_channel, relu, 1, M, N, K,

@@ -262,6 +262,42 @@ def test_raw_accumulator_readout_and_split_k(M, N, K, ldd_pad):
     i8.set_path(0)
 
 
+@pytest.mark.parametrize("M,N,K,lda_pad,ldb_pad,b_row_major", [(300, 200, 100, 3, 7, 0), (512, 384, 250, 0, 0, 1), (777, 130, 64, 5, 2, 1)])
+def test_raw_and_float_scale_readouts_on_packed_operands(M, N, K, lda_pad, ldb_pad, b_row_major):
+    """The other two read-outs with operands the tensor path cannot fetch in place (odd leading dimensions, K that is not a
+    multiple of 16; for the float scale also row-major B): packed copies, tensor kernels, same results as the oracle."""
+    import torch
+    import oracle
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_gemm(M, N, K, 4900 + M + K, per_channel=1, relu=1, lda_pad=lda_pad, ldb_pad=ldb_pad)
+    acc = oracle.gemm_acc(p.A, p.a_rs, 1, p.B, 1, p.b_cs, M, N, K).astype(np.int32)
+    rng = np.random.default_rng(M)
+    scale = (rng.uniform(0.5, 1.0, size=N) * 2.0 ** rng.integers(-13, -9, size=N)).astype(np.float32)
+    want_f = oracle.gemm_i8_fscale(p.A, p.a_rs, 1, p.B, 1, p.b_cs, N, p.bias, scale, 1, M, N, K, 1)
+    A = torch.from_numpy(p.A).cuda()[:, :K]
+    Bk = torch.from_numpy(p.B).cuda()[:, :K]                                  # (N, K) storage, K contiguous
+    Bn = torch.from_numpy(np.ascontiguousarray(p.B[:, :K].T)).cuda()          # (K, N) storage, N contiguous
+    bias, sc = torch.from_numpy(p.bias).cuda(), torch.from_numpy(scale).cuda()
+    for mode in (0, 1):
+        i8.set_path(mode)
+        D = torch.full((M, N), 77, dtype=torch.int32, device="cuda")
+        i8.gemm_i8_raw(A, Bk.t(), D)
+        if (lda_pad or ldb_pad or K % 16) and mode == 0:
+            assert i8.last_gemm_packed() and i8.last_path() in TENSOR_PATHS, (i8.last_gemm_packed(), i8.last_path())
+        H.assert_same(D.cpu().numpy(), acc, f"raw, packed, mode {mode}")
+        C = torch.full((M, N), 0x5A, dtype=torch.int8, device="cuda")
+        i8.gemm_i8_fscale(A, Bn if b_row_major else Bk.t(), C, bias, sc, 1, 1)
+        if mode == 0:
+            assert i8.last_gemm_packed() == bool(b_row_major or lda_pad or ldb_pad or K % 16)
+            assert i8.last_path() in TENSOR_PATHS, i8.last_path()
+        else:
+            assert i8.last_path() == i8.PATH_GENERIC
+        H.assert_same(C.cpu().numpy(), want_f, f"float scale, packed, mode {mode}")
+        assert i8.last_device_status() == 0
+    i8.set_path(0)
+    H.not_degenerate(want_f)
+
+
 @pytest.mark.parametrize("M,N,K", [(512, 512, 128), (513, 600, 1040), (1000, 520, 272), (640, 1300, 144), (769, 1025, 48), (2048, 1536, 4096),
                                    (100, 300, 64), (256, 64, 96)])
 def test_two_sm_kernel_shapes(M, N, K):
