@@ -360,6 +360,7 @@ def main():
             time.sleep(0.5)             # the per-configuration timings start from an idle GPU, not from the power-capped clock
             details = bench_details.run(dev, peak_tops=2 * pk["bf16_burst"], peak_gbs=pk["hbm_gbs"], oracle=oracle_t)
         # this library's own tensor-core issue-rate probe (operands resident in shared memory): burst and sustained
+        time.sleep(0.5)                 # the burst figure is taken from an idle GPU as well
         probe = bench_details.run_peak(dev)
 
     if rank == 0:
