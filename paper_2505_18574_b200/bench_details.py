@@ -1,5 +1,6 @@
 """Per-problem timings of every workload configuration (GEMM 256^3, the three large GEMMs, the four
-convolutions, the tall-skinny GEMM and the batched 64^3 products; `--cfg mpc` adds the fp32 TinyMPC forward pass over
+convolutions, the tall-skinny GEMM and the batched 64^3 products, a batch of 128^3 products, a 4096^3 GEMM with row-major
+B; `--cfg mpc` adds the fp32 TinyMPC forward pass over
 2^20 instances, `--cfg sweep` the shapes the paper prints, `--cfg peak` the tensor-core issue-rate probe that gives the
 int8 roofline its measured denominator) through the C-ABI binding.
 
@@ -24,7 +25,7 @@ import numpy as np
 # Order of a full run: the microsecond kernels first, the three large GEMMs last.  Those run for milliseconds at the power
 # cap, and the lowered clock outlasts them: timed right behind them, the 56 x 56 convolution measured 11-13 us against
 # 9.1 us from an idle GPU, the next configuration 8.4 against 7.3, the ones after that unchanged.
-ALL = ["0", "2", "3a", "3b", "3c", "4a", "4b", "mpc", "1a", "1b", "1c"]
+ALL = ["0", "2", "3a", "3b", "3c", "4a", "4b", "b128", "mpc", "rmB", "1a", "1b", "1c"]
 # the shapes the paper prints: "g0".."g9" (inputs.SWEEP_GEMMS) and "c0", "c1" (inputs.SWEEP_CONVS)
 SWEEP = [f"g{i}" for i in range(10)] + ["c0", "c1"]
 L2_BYTES = 126e6
@@ -34,6 +35,10 @@ def _problem(name):
     from . import inputs
     if name == "mpc":
         return inputs.make_mpc(1 << 20)
+    if name == "rmB":
+        return inputs.extra_rowmajor_b()
+    if name == "b128":
+        return inputs.extra_batched_128()
     if name[0] == "g":
         return inputs.sweep_gemm(int(name[1:]))
     if name[0] == "c":
@@ -62,7 +67,8 @@ def _make(name, dev, copies_for_l2=True):
         calls = []
         for _ in range(sets):
             A, B, C = T(p.A), T(p.B), torch.empty((p.M, p.N), dtype=torch.int8, device=dev)
-            calls.append(i8.prepare("gemm_i8", A, B.t(), C, b, mu, sh, p.per_channel, p.relu))
+            Bv = B.t() if p.b_rs == 1 else B           # logical (K, N): stored (N, K) K-contiguous, or row-major as it is
+            calls.append(i8.prepare("gemm_i8", A, Bv, C, b, mu, sh, p.per_channel, p.relu))
     elif isinstance(p, inputs.ConvProblem):
         ops = 2.0 * p.N * p.P * p.Q * p.K * p.R * p.S * p.C
         byts = p.x.size + p.w.size + p.N * p.P * p.Q * p.K + 12 * p.K

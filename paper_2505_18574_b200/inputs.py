@@ -203,6 +203,16 @@ def config4b() -> BatchedProblem:
     return make_batched(16384, 64, 64, 64, 104, name="cfg4b_batched_16384x64")
 
 
+def extra_rowmajor_b() -> GemmProblem:
+    """4096^3 with B stored row-major [K][N], the layout of the paper's printed Gemmini GEMM listing; otherwise as config 1a."""
+    return make_gemm(4096, 4096, 4096, 501, b_layout="row", per_channel=1, relu=0, name="extra_gemm_4096cube_rowmajorB")
+
+
+def extra_batched_128() -> BatchedProblem:
+    """256 independent 128^3 products (above the paired 64^3 tile: one launch of the large-tile kernel per problem)."""
+    return make_batched(256, 128, 128, 128, 502, name="extra_batched_256x128cube")
+
+
 # ---------------------------------------------------------------------------------------------
 # Shapes the paper itself prints (second workload): the Gemmini GEMM of its Code Examples
 # appendix, the schedule-reuse table (square / column-dominant / row-dominant GEMMs, read as
