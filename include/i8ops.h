@@ -129,6 +129,10 @@ int gemm_i8_fscale(const int8_t* A, int64_t a_rs, int64_t a_cs,
  * products, Evaluation "Fine-Grained Linear Algebra"; also its column-dominant GEMM shapes).
  * Problem b uses A + b*a_bs, B + b*b_bs, C + b*c_bs and bias + b*bias_bs (bias_bs == 0: one bias
  * shared by all problems); mult/shift are shared by all problems.  Other arguments as gemm_i8.
+ * Kernels: problems up to 64 x 64 x 64 run two to an instruction on the paired small-tile kernel; larger ones with
+ * 16-byte aligned slices run in ONE launch of the large-tile kernel whose tile schedule covers all problems (row-major
+ * A, either storage order of B, batch strides that are whole rows), else one launch per problem, else the
+ * one-thread-per-output kernel.  Same results on every path.
  * Errors as gemm_i8, plus I8_ERR_SHAPE for a negative batch.
  */
 int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs,

@@ -169,8 +169,9 @@ struct TmapEntry {
     alignas(64) CUtensorMap map;
     bool valid;
 };
-constexpr int TMAP_CACHE_SLOTS = 64;
-static thread_local TmapEntry t_tmap_cache[TMAP_CACHE_SLOTS];
+constexpr int TMAP_CACHE_SETS = 32, TMAP_CACHE_WAYS = 4;      // four ways: the two or three maps of one call never evict each other
+static thread_local TmapEntry t_tmap_cache[TMAP_CACHE_SETS][TMAP_CACHE_WAYS];
+static thread_local uint8_t t_tmap_next[TMAP_CACHE_SETS];     // way to replace next, per set
 static thread_local uint64_t t_tmap_hits = 0, t_tmap_misses = 0;
 
 static uint32_t tmap_hash(const TmapKey& k) {
@@ -200,15 +201,20 @@ static int encode_tmap(CUtensorMap* tm, const TmapKey& k) {
 
 static int cached_tmap(CUtensorMap* tm, const TmapKey& k) {
     if (!g_tmap_cache) return encode_tmap(tm, k);
-    TmapEntry& e = t_tmap_cache[tmap_hash(k) % TMAP_CACHE_SLOTS];
-    if (e.valid && memcmp(&e.key, &k, sizeof(TmapKey)) == 0) {
-        *tm = e.map;
-        t_tmap_hits++;
-        return I8_OK;
+    const uint32_t set = tmap_hash(k) % TMAP_CACHE_SETS;
+    for (int w = 0; w < TMAP_CACHE_WAYS; w++) {
+        const TmapEntry& e = t_tmap_cache[set][w];
+        if (e.valid && memcmp(&e.key, &k, sizeof(TmapKey)) == 0) {
+            *tm = e.map;
+            t_tmap_hits++;
+            return I8_OK;
+        }
     }
     t_tmap_misses++;
     int rc = encode_tmap(tm, k);
     if (rc) return rc;
+    TmapEntry& e = t_tmap_cache[set][t_tmap_next[set]];
+    t_tmap_next[set] = (uint8_t)((t_tmap_next[set] + 1) % TMAP_CACHE_WAYS);
     e.key = k; e.map = *tm; e.valid = true;
     return I8_OK;
 }
@@ -431,10 +437,14 @@ static TcPlan plan_tc(bool conv, int M, int N, int K, int num_kb, int num_iters,
 // Common tail of the tensor paths: B's tensor map (an N x K matrix with K contiguous), the tile schedule,
 // and the launch of the instance that matches the tile width.
 struct RawOut { int32_t* D = nullptr; int64_t ldd = 0; int accumulate = 0; };
+// Independent problems of one shape in one launch: problem b starts a_rpp / b_rpp / c_rpp rows further in the stacked
+// 2-D views of A / B / C, its bias bias_bs entries further; mt = block rows per problem.
+struct BatchInfo { int batch = 1, mt = 0; int64_t a_rpp = 0, b_rpp = 0, c_rpp = 0, bias_bs = 0; };
 
 static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap& tmA, const KLoop& kl, const int8_t* B,
                   int64_t ldb, int8_t* C, int64_t ldc, const int32_t* bias, const int32_t* mult, const int32_t* shift,
-                  int per_channel, int M, int N, int K, int relu, cudaStream_t st, const RawOut& raw = RawOut()) {
+                  int per_channel, int M, int N, int K, int relu, cudaStream_t st, const RawOut& raw = RawOut(),
+                  const BatchInfo& bt = BatchInfo()) {
     const bool two_sm = pl.two_sm != 0;
     const int bn = pl.bn;
     const int b_rows = two_sm ? bn / 2 : bn;           // rows of the B tile one CTA loads
@@ -444,19 +454,22 @@ static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap
     if (kl.b_mn) {
         // B stored with N contiguous: K rows of 128 (64-wide tiles: 64) bytes of N
         const uint32_t mnw = b_rows >= 128 ? 128u : 64u;
-        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)K};
+        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)((bt.batch - 1) * bt.b_rpp + K)};
         const uint64_t str[1] = {(uint64_t)ldb};
         const uint32_t box[2] = {mnw, (uint32_t)BK};
         int rc = make_tmap(&tmB, B, 2, dims, str, box, mnw == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
         if (rc) return rc;
     } else {
-        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)((bt.batch - 1) * bt.b_rpp + N)};
         const uint64_t str[1] = {(uint64_t)ldb};
         const uint32_t box[2] = {(uint32_t)kl.cb, (uint32_t)b_rows};
         int rc = make_tmap(&tmB, B, 2, dims, str, box, swizzle_for(kl.cb));
         if (rc) return rc;
     }
     GemmTcParams p;
+    p.batch_mt = bt.batch > 1 ? bt.mt : 0;
+    p.inv_bmt = bt.mt <= 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)bt.mt);
+    p.a_rpp = (int)bt.a_rpp; p.b_rpp = (int)bt.b_rpp; p.c_rpp = bt.c_rpp; p.bias_bs = bt.batch > 1 ? bt.bias_bs : 0;
     p.C = C; p.ldc = ldc; p.bias = bias; p.mult = mult; p.shift = shift;
     p.per_channel = per_channel; p.relu = relu; p.M = M; p.N = N; p.K = K;
     p.c_vec_ok = raw.D ? (aligned16(raw.D) && raw.ldd % 4 == 0) : (aligned16(C) && (ldc % 16 == 0));
@@ -466,7 +479,7 @@ static int run_tc(DeviceCtx* ctx, bool conv, const TcPlan& pl, const CUtensorMap
     // it would write up to 15 bytes past the last column
     CUtensorMap tmC = tmB;
     p.tma_store = 0;
-    if (g_tma_store && !raw.D && bn >= 128 && p.c_vec_ok && N % 16 == 0) {
+    if (g_tma_store && !raw.D && bn >= 128 && p.c_vec_ok && N % 16 == 0 && bt.batch == 1) {
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)M};
         const uint64_t str[1] = {(uint64_t)ldc};
         const uint32_t box[2] = {64, 32};
@@ -550,6 +563,42 @@ static int run_gemm_tc(DeviceCtx* ctx, const int8_t* A, int64_t lda, const int8_
     int rc = make_tmap(&tmA, A, 2, a_mn ? dims_m : dims_k, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
     return run_tc(ctx, false, pl, tmA, kl, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, raw);
+}
+
+// A batch of equal-shape problems (K-contiguous operands, batch strides that are whole numbers of rows) as ONE launch of
+// the large-tile kernel on single CTAs: the tile schedule runs over the block rows of all problems.
+static int run_gemm_tc_batched(DeviceCtx* ctx, const int8_t* A, int64_t lda, int64_t a_bs, const int8_t* B, int64_t ldb, int64_t b_bs,
+                               int8_t* C, int64_t ldc, int64_t c_bs, const int32_t* bias, int64_t bias_bs, const int32_t* mult,
+                               const int32_t* shift, int per_channel, int batch, int M, int N, int K, int relu, cudaStream_t st,
+                               int b_mn) {
+    if (a_bs % lda || b_bs % ldb || c_bs % ldc) return I8_ERR_UNSUPPORTED;
+    BatchInfo bt;
+    bt.batch = batch; bt.a_rpp = a_bs / lda; bt.b_rpp = b_bs / ldb; bt.c_rpp = c_bs / ldc; bt.bias_bs = bias_bs;
+    bt.mt = (M + BM - 1) / BM;
+    const int64_t rows_a = (batch - 1) * bt.a_rpp + M, rows_b = (batch - 1) * bt.b_rpp + (b_mn ? K : N);
+    if (rows_a >= (1ll << 31) - BM || rows_b >= (1ll << 31) - 256 || (int64_t)bt.mt * batch >= (1ll << 24)) return I8_ERR_UNSUPPORTED;
+    KLoop kl = gemm_kloop(K);
+    kl.b_mn = b_mn;
+    TcPlan pl = {};
+    pl.shape_cls = shape_class(M, N);
+    pl.two_sm = 0;
+    pl.bn = choose_bn((int)((int64_t)bt.mt * batch > 65536 ? 65536 * BM : bt.mt * batch * BM), N, kl.num_kblocks, ctx->sm_count, nullptr);
+    pl.tile_m = BM;
+    pl.stages = pl.bn == 256 ? 4 : 6;
+    pl.m_tiles = bt.mt * batch;
+    pl.n_tiles = (N + pl.bn - 1) / pl.bn;
+    if ((int64_t)pl.m_tiles * pl.n_tiles >= (1ll << 30)) return I8_ERR_UNSUPPORTED;
+    pl.num_tiles = pl.m_tiles * pl.n_tiles;
+    pl.workers = pl.num_tiles < ctx->sm_count ? pl.num_tiles : ctx->sm_count;
+    pl.group_m = 16;
+    pl.sticky = 0; pl.col_base = 0; pl.col_rem = 0; pl.b_resident = 0;
+    CUtensorMap tmA;
+    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)rows_a};
+    const uint64_t str[1] = {(uint64_t)lda};
+    const uint32_t box[2] = {BK, BM};
+    int rc = make_tmap(&tmA, A, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    return run_tc(ctx, false, pl, tmA, kl, B, ldb, C, ldc, bias, mult, shift, per_channel, M, N, K, relu, st, RawOut(), bt);
 }
 
 // ------------------------------------------------------------------------------------------------ channel-major kernel
@@ -1168,24 +1217,34 @@ int batched_gemm_i8(const int8_t* A, int64_t a_rs, int64_t a_cs, int64_t a_bs, c
             if (!(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
         }
     }
-    // Larger problems: one launch of the large-tile (or channel-major) kernel per problem, when each problem is big enough
-    // to be worth a launch of its own (128^3 multiply-accumulates, or a short batch) and every slice keeps the alignment
-    // the tensor path needs.
-    if (g_path_mode != 1 && K >= 1 && ((int64_t)M * N * K >= (1ll << 21) || batch <= 8) && batch <= 65536) {
+    // Larger problems with aligned slices.  All problems in ONE launch of the large-tile kernel when A is K-contiguous and
+    // the batch strides are whole rows (the tile schedule runs over the stacked problems); otherwise one launch per
+    // problem, when each problem is big enough to be worth a launch of its own (128^3 multiply-accumulates, or a short
+    // batch).
+    if (g_path_mode != 1 && K >= 1 && batch <= 65536) {
         const bool a_k = a_cs == 1 && a_rs % 16 == 0 && a_rs >= K, a_m = !a_k && a_rs == 1 && a_cs % 16 == 0 && a_cs >= M;
         const bool b_k = b_rs == 1 && b_cs % 16 == 0 && b_cs >= K, b_n = !b_k && b_cs == 1 && b_rs % 16 == 0 && b_rs >= N;
         if (aligned16(A) && aligned16(B) && a_bs % 16 == 0 && b_bs % 16 == 0 && (a_k || a_m) && (b_k || b_n)) {
-            int last = I8_PATH_NONE;
-            for (int b = 0; b < batch; b++) {
-                t_used_two_sm = false; t_tmap_failed = false;
-                rc = run_gemm_tc(ctx, A + (int64_t)b * a_bs, a_k ? a_rs : a_cs, B + (int64_t)b * b_bs, b_k ? b_cs : b_rs, C + (int64_t)b * c_bs, ldc,
-                                 bias ? bias + (int64_t)b * bias_bs : nullptr, mult, shift, per_channel, M, N, K, relu, st, RawOut(),
-                                 a_m ? 1 : 0, b_n ? 1 : 0);
-                if (rc == I8_ERR_CUDA && t_tmap_failed && b == 0) break;        // no tensor map for this geometry: generic kernel below
-                if (rc) return rc;
-                last = tensor_path_used();
+            if (batch > 1 && a_k && a_bs > 0 && b_bs > 0 && c_bs > 0) {
+                t_used_two_sm = false; t_tmap_failed = false; t_used_swap = false;
+                rc = run_gemm_tc_batched(ctx, A, a_rs, a_bs, B, b_k ? b_cs : b_rs, b_bs, C, ldc, c_bs, bias, bias_bs, mult, shift,
+                                         per_channel, batch, M, N, K, relu, st, b_n ? 1 : 0);
+                if (rc == I8_OK) { t_last_path = tensor_path_used(); return rc; }
+                if (rc != I8_ERR_UNSUPPORTED && !(rc == I8_ERR_CUDA && t_tmap_failed)) return rc;
             }
-            if (rc == I8_OK) { t_last_path = last; return rc; }
+            if ((int64_t)M * N * K >= (1ll << 21) || batch <= 8) {
+                int last = I8_PATH_NONE;
+                for (int b = 0; b < batch; b++) {
+                    t_used_two_sm = false; t_tmap_failed = false;
+                    rc = run_gemm_tc(ctx, A + (int64_t)b * a_bs, a_k ? a_rs : a_cs, B + (int64_t)b * b_bs, b_k ? b_cs : b_rs, C + (int64_t)b * c_bs, ldc,
+                                     bias ? bias + (int64_t)b * bias_bs : nullptr, mult, shift, per_channel, M, N, K, relu, st, RawOut(),
+                                     a_m ? 1 : 0, b_n ? 1 : 0);
+                    if (rc == I8_ERR_CUDA && t_tmap_failed && b == 0) break;        // no tensor map for this geometry: generic kernel below
+                    if (rc) return rc;
+                    last = tensor_path_used();
+                }
+                if (rc == I8_OK) { t_last_path = last; return rc; }
+            }
         }
     }
     GenericGemmParams g{A, a_rs, a_cs, a_bs, B, b_rs, b_cs, b_bs, C, ldc, c_bs, bias, bias_bs, mult, shift, per_channel, relu,

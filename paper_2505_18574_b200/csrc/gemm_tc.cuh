@@ -108,6 +108,14 @@ struct GemmTcParams {
     int raw, accumulate;        // raw != 0 selects D; accumulate != 0 adds to what D already holds
     TileSched sched;
     KLoop kl;
+    // Independent problems of one shape in one launch (batch_mt != 0): the operands are read as matrices of stacked
+    // problems, problem b starting a_rpp / b_rpp / c_rpp rows further in A / B / C, and the schedule's block rows run
+    // over all problems (batch_mt block rows each).  Rows of a tile beyond M belong to the next problem in A and are
+    // never stored; the bias of problem b starts bias_bs entries further.
+    int batch_mt;
+    uint32_t inv_bmt;           // floor(2^32 / batch_mt)
+    int a_rpp, b_rpp;
+    int64_t c_rpp, bias_bs;
     long long wait_limit_cycles;
     unsigned* dev_status;
 };
@@ -357,8 +365,15 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int tile = first_tile; ok && tile < tile_end; tile += tile_step) {
             int m_blk, n_blk;
             sched.map(tile, first_tile, tile_step, m_blk, n_blk);
-            const int row_a = m_blk * TILE_M + (int)rank * BM;          // this CTA's first A row (output row / pixel)
-            const int row_b = n_blk * BN + (int)rank * B_ROWS;          // this CTA's first B row (output column)
+            int prob = 0;                                               // which of the stacked problems
+            if (p.batch_mt) { prob = fast_div(m_blk, p.batch_mt, p.inv_bmt); m_blk -= prob * p.batch_mt; }
+            const int row_a = prob * p.a_rpp + m_blk * TILE_M + (int)rank * BM;   // this CTA's first A row (output row / pixel)
+            // this CTA's first B row (output column); a stacked problem starts b_rpp rows further: rows of N for K-major B,
+            // rows of K for MN-major B (where a ragged last K block then reads the next problem's rows: they meet the
+            // zeros that A's own K edge is filled with)
+            const int b_mn_now = !CONV && kl.b_mn;
+            const int row_b = (b_mn_now ? 0 : prob * p.b_rpp) + n_blk * BN + (int)rank * B_ROWS;
+            const int k_off_b = b_mn_now ? prob * p.b_rpp : 0;
             int w0 = 0, h0 = 0, img = 0;
             if (CONV) {
                 // first output pixel of the tile -> position of filter tap (0,0) in the input image
@@ -405,8 +420,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                             constexpr int NBOX = B_ROWS > 128 ? B_ROWS / 128 : 1;
 #pragma unroll
                             for (int h = 0; h < NBOX; h++) {
-                                if (TWO_SM) tma_load_2d_pair(dstB + h * (128 * BK), &tmB, full, row_b + h * 128, kbi * BK);
-                                else tma_load_2d(dstB + h * (128 * BK), &tmB, full, row_b + h * 128, kbi * BK);
+                                if (TWO_SM) tma_load_2d_pair(dstB + h * (128 * BK), &tmB, full, row_b + h * 128, k_off_b + kbi * BK);
+                                else tma_load_2d(dstB + h * (128 * BK), &tmB, full, row_b + h * 128, k_off_b + kbi * BK);
                             }
                         } else {
                             if (TWO_SM) tma_load_2d_pair(dstB, &tmB, full, kbi * kl.cb, row_b);
@@ -522,8 +537,11 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int tile = first_tile; tile < tile_end; tile += tile_step) {
             int m_blk, n_blk;
             sched.map(tile, first_tile, tile_step, m_blk, n_blk);
+            int prob = 0;
+            if (p.batch_mt) { prob = fast_div(m_blk, p.batch_mt, p.inv_bmt); m_blk -= prob * p.batch_mt; }
             const int n0 = n_blk * BN;
-            if (n_blk != cached_n_blk) {
+            const int col_key = p.bias_bs ? n_blk + prob * sched.n_tiles : n_blk;   // a per-problem bias: new constants per problem
+            if (col_key != cached_n_blk) {
                 // new block column: rebuild the per-channel constants (before waiting, so this overlaps the main loop)
                 named_barrier(1, EPI_THREADS);            // nobody still reads the previous column's constants
                 bool all32 = true, allfold = true;
@@ -531,7 +549,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const int n = n0 + c;
                     int32_t bias = 0, mult = 0, shift = 0;
                     if (n < p.N && !p.raw) {
-                        bias = p.bias ? p.bias[n] : 0;
+                        bias = p.bias ? p.bias[(int64_t)prob * p.bias_bs + n] : 0;
                         mult = p.mult[p.per_channel ? n : 0];
                         shift = p.shift[p.per_channel ? n : 0];
                     }
@@ -545,7 +563,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     s_m2[c] = m2;
                     s_c64[c] = make_fold_addend(bias, m2);
                 }
-                cached_n_blk = n_blk;
+                cached_n_blk = col_key;
                 shift32 = named_barrier_and(2, EPI_THREADS, all32);
                 fold = named_barrier_and(3, EPI_THREADS, allfold);
                 if constexpr (ONE_CHUNK) if (fold) {
@@ -560,7 +578,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (dead) continue;
             tc_fence_after();
             const int row = m_blk * TILE_M + (int)rank * BM + quarter * 32 + lane;
-            int8_t* crow = p.C + (int64_t)row * p.ldc;
+            int8_t* crow = p.C + ((int64_t)prob * p.c_rpp + row) * p.ldc;
             const uint32_t t0 = tmem_base + ab * BN + ((uint32_t)(quarter * 32) << 16);
             // staging buffer of this warp: row r holds four 16-byte units, unit u at position u ^ ((r >> 1) & 3) (the
             // 64-byte TMA swizzle, which also keeps the row-wise 16-byte writes free of bank conflicts)

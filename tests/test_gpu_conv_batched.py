@@ -289,8 +289,8 @@ def test_batched_shapes(batch, M, N, K, ppb):
 
 @pytest.mark.parametrize("batch,M,N,K", [(3, 128, 128, 128), (5, 256, 192, 320), (2, 130, 144, 80), (40, 128, 128, 128), (4, 1024, 512, 256)])
 def test_batched_problems_larger_than_the_paired_tile(batch, M, N, K):
-    """Problems above 64 in any dimension: one launch of the large-tile kernel per problem (row-major B through the MN-major
-    descriptor), per-problem bias."""
+    """Problems above 64 in any dimension on the large-tile kernel (row-major B through the MN-major descriptor), per-problem
+    bias."""
     import paper_2505_18574_b200 as i8
     p = inputs.make_batched(batch, M, N, K, 700 + batch + M + N)
     p.shift[:] = 24
@@ -299,6 +299,41 @@ def test_batched_problems_larger_than_the_paired_tile(batch, M, N, K):
     got = H.batched_gpu(p)
     assert i8.last_path() in (i8.PATH_TENSOR, i8.PATH_TENSOR_2SM, i8.PATH_CHANNEL_MAJOR, i8.PATH_CHANNEL_MAJOR_2SM), i8.last_path()
     H.assert_same(got, want, p.name)
+    H.not_degenerate(want)
+
+
+@pytest.mark.parametrize("batch,M,N,K,ppb", [(6, 200, 144, 96, True), (300, 96, 80, 112, True), (17, 128, 304, 272, False),
+                                             (64, 128, 128, 128, True), (9, 65, 16, 1040, True)])
+@pytest.mark.parametrize("b_col_major", [False, True])
+def test_batched_problems_in_one_launch(batch, M, N, K, ppb, b_col_major):
+    """Problems above the paired 64^3 tile, all in one launch of the large-tile kernel: the tile schedule runs over the
+    stacked problems (block rows of A that cross into the next problem are never stored), either storage order of B,
+    per-problem and shared bias, a padded batch stride of C whose gaps must stay untouched."""
+    import torch
+    import paper_2505_18574_b200 as i8
+    p = inputs.make_batched(batch, M, N, K, 800 + batch + M + N + K, per_problem_bias=ppb)
+    p.shift[:] = 22
+    want = H.batched_oracle(p)
+    A = torch.from_numpy(p.A).cuda()
+    if b_col_major:
+        B = torch.from_numpy(np.ascontiguousarray(p.B.transpose(0, 2, 1))).cuda().transpose(1, 2)   # (batch, K, N) view, K contiguous
+    else:
+        B = torch.from_numpy(p.B).cuda()
+    Cbuf = torch.full((batch, M + 3, N), 0x5A, dtype=torch.int8, device="cuda")                      # three spare rows per problem
+    C = Cbuf[:, :M, :]
+    bias, mult, shift = (torch.from_numpy(v).cuda() for v in (p.bias, p.mult, p.shift))
+    for mode in (0, 1):
+        i8.set_path(mode)
+        Cbuf.fill_(0x5A)
+        i8.batched_gemm_i8(A, B, C, bias, mult, shift, p.per_channel, p.relu)
+        assert i8.last_device_status() == 0
+        assert (i8.last_path() == i8.PATH_TENSOR) if mode == 0 else (i8.last_path() == i8.PATH_GENERIC), i8.last_path()
+        H.assert_same(C.cpu().numpy(), want, f"{p.name} mode {mode} b_col_major={b_col_major}")
+        assert (Cbuf[:, M:, :] == 0x5A).all(), "rows between the problems of C were written"
+    if batch > 8:
+        plan = i8.last_plan()        # generic mode ran last: the plan still shows the tensor launch before it
+        assert plan["m_tiles"] == batch * ((M + 127) // 128), plan
+    i8.set_path(0)
     H.not_degenerate(want)
 
 
